@@ -1,0 +1,363 @@
+"""Pins for the CPU oracle: every part of it is held to something other than itself --
+values the paper prints, closed forms, brute force, a library cast, fp64 attention."""
+import ctypes as C
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import lamp_inputs as li
+import oracle
+
+L = oracle.lib()
+GOLD = {}
+for line in open(os.path.join(os.path.dirname(__file__), "golden", "paper_constants.txt")):
+    line = line.split("#")[0].strip()
+    if "=" in line:
+        k, v = [s.strip() for s in line.split("=")]
+        GOLD[k] = float(int(v, 16)) if v.startswith("0x") else float(v)
+
+E4M3_GRID = sorted({float(L.lamp_oracle_dec_e4m3(b)) for b in range(256) if (b & 0x7F) != 0x7F})
+
+
+def brute_nearest_even(x, grid):
+    """Nearest grid value by exhaustive search; a tie goes to the value whose index in the
+    (uniformly coded) grid is even -- grids here start at 0 with index 0."""
+    best = min(range(len(grid)), key=lambda i: (abs(grid[i] - x), i % 2))
+    return grid[best]
+
+
+# ---------------------------------------------------------------- P1: e4m3 rounding
+
+def test_e4m3_grid_matches_format_definition():
+    pos = [g for g in E4M3_GRID if g >= 0]
+    assert len(pos) == 127 and pos[0] == 0.0
+    assert pos[-1] == GOLD["e4m3_max"]                      # Sec. 3.3: limit 448
+    assert pos[1] == 2.0 ** -9 and pos[8] == 2.0 ** -6      # subnormal quantum, min normal
+    for b in range(256):
+        if (b & 0x7F) == 0x7F:
+            continue
+        v = L.lamp_oracle_dec_e4m3(b)
+        assert L.lamp_oracle_enc_e4m3(v) == (0 if b == 0x80 else b)
+
+
+@pytest.mark.parametrize("x,want", [(17, 16), (19, 20), (21, 20), (100, 96), (0.3, 0.3125),
+                                    (-5.3, -5.5), (2.0 ** -10, 0.0), (3 * 2.0 ** -10, 2.0 ** -8),
+                                    (463.9, 448), (464, 448), (1e9, 448), (-1e9, -448),
+                                    (447.9, 448), (2.0 ** -9 * 0.51, 2.0 ** -9)])
+def test_e4m3_worked_values(x, want):
+    assert L.lamp_oracle_rne_e4m3(x) == want
+
+
+def test_e4m3_against_brute_force_and_torch_cast():
+    rng = np.random.default_rng(0)
+    xs = np.concatenate([rng.normal(0, 30, 4000), rng.normal(0, 0.02, 2000),
+                         rng.uniform(-470, 470, 2000),
+                         np.array([(a + b) / 2 for a, b in zip(E4M3_GRID[:-1], E4M3_GRID[1:])])])
+    xs = xs.astype(np.float32)
+    got = np.array([L.lamp_oracle_rne_e4m3(float(x)) for x in xs], np.float32)
+    pos = [g for g in E4M3_GRID if g >= 0]
+    for x, g in zip(xs[::7], got[::7]):
+        w = math.copysign(brute_nearest_even(min(abs(float(x)), 448.0), pos), float(x))
+        assert g == w, (x, g, w)
+    inr = np.abs(xs) <= 448
+    lib = torch.from_numpy(xs[inr]).to(torch.float8_e4m3fn).to(torch.float32).numpy()
+    assert np.array_equal(lib, got[inr])
+
+
+def test_e4m11_and_truncation():
+    # e4m11: 12 significant bits, same exponent range, max 448
+    assert L.lamp_oracle_rne_e4m11(1.0 + 2.0 ** -12) == 1.0            # tie -> even
+    assert L.lamp_oracle_rne_e4m11(1.0 + 3 * 2.0 ** -12) == 1.0 + 2.0 ** -10
+    assert L.lamp_oracle_rne_e4m11(300.06) == 300.0                    # quantum 2^-3 at [256, 512)
+    assert L.lamp_oracle_rne_e4m11(2.0 ** -18 * 1.01) == 2.0 ** -17    # subnormal quantum 2^-17
+    assert L.lamp_oracle_rne_e4m11(1e5) == 448.0 and L.lamp_oracle_rne_e4m11(-449.0) == -448.0
+    for x, w in [(31.9, 30.0), (3.3, 3.25), (-5.3, -5.0), (448.0, 448.0),
+                 (2.0 ** -7 + 2.0 ** -17, 2.0 ** -7)]:
+        x16 = L.lamp_oracle_rne_e4m11(x)
+        t = L.lamp_oracle_trunc_e4m3(x16)
+        assert t == w and t in E4M3_GRID and abs(t) <= abs(x16)
+
+
+# ------------------------------------------------- P2: accumulation order and tie rule
+
+def chain(a, b):
+    a = np.asarray(a, np.float32); b = np.asarray(b, np.float32)
+    return L.lamp_oracle_chain8(a.ctypes.data_as(C.c_void_p), b.ctypes.data_as(C.c_void_p), len(a))
+
+
+def test_chain_swamping_examples():
+    assert chain([1.0] * 128, [1.0] * 128) == 16.0        # 16 + 1 = 17 ties back to 16
+    assert chain([0.75] * 128, [1.0] * 128) == 16.0       # exact sum 96
+    assert chain([1.0, -0.5] * 64, [1.0] * 128) == 7.5    # exact sum 32
+    # order matters: the large term first swallows the small ones, last it does not
+    assert chain([64.0] + [1.0] * 16, [1.0] * 17) == 64.0
+    assert chain([1.0] * 16 + [64.0], [1.0] * 17) == 80.0
+    # one rounding per step, fused: 3 * 1.4375 + 0.3125 = 4.625 -> tie -> 4.5; an unfused
+    # product rounded first (4.3125 -> no such step exists) would differ in other cases
+    assert chain([3.0, 1.4375], [0.1041666716337204, 3.0]) == L.lamp_oracle_rne_e4m3(
+        float(np.float32(np.float64(np.float32(1.4375)) * 3.0 + 0.3125)))
+
+
+def test_overflow_rule_of_section_3_3():
+    f = GOLD["logit_bound_factor"]
+    assert abs(f - 8 * math.sqrt(2)) < 1e-12
+    assert f * GOLD["maxgain_ok"] ** 2 <= GOLD["e4m3_max"] < f * 6.30 ** 2
+    # the bound is reached by an RMS-normalised row times the gain on both sides, with the
+    # 1/sqrt(d) scale folded into q: 128 equal terms g*g/sqrt(128) never exceed 448
+    g = np.float32(GOLD["maxgain_ok"])
+    qs = np.full(128, g / np.float32(math.sqrt(128)), np.float32)
+    assert chain(np.full(128, g, np.float32), qs) <= 448.0
+
+
+# ------------------------------------------------------------ P4/P5: exponential formats
+
+def test_exponential_format_constants():
+    assert L.lamp_oracle_dec_exp8(int(GOLD["exp_one_pattern"])) == 1.0
+    assert L.lamp_oracle_dec_exp8(0x08) == 2.0 ** GOLD["exp_min_normal_log2"]
+    assert L.lamp_oracle_dec_exp8(0x01) == 2.0 ** GOLD["exp_min_subnormal_log2"]
+    assert L.lamp_oracle_dec_ue5m3(L.lamp_oracle_enc_ue5m3(GOLD["shift_max"])) == GOLD["shift_max"]
+    for p in range(8, 256):
+        assert L.lamp_oracle_enc_ue5m3(L.lamp_oracle_dec_ue5m3(p)) == p
+
+
+def test_lut8_is_the_correctly_rounded_exponential():
+    grid = [L.lamp_oracle_dec_exp8(b) for b in range(0xF9)]      # 0 .. 1.0, index = byte
+    nonzero = 0
+    prev = 0xF8
+    for p in range(256):
+        s = L.lamp_oracle_dec_ue5m3(p)
+        got = L.lamp_oracle_lut8(p)
+        want = brute_nearest_even(math.exp(-s), grid)
+        assert L.lamp_oracle_dec_exp8(got) == want, (p, s)
+        if s >= 2.0 ** -9 and s <= 896:
+            assert got <= prev
+            prev = got
+            nonzero += got != 0
+    assert nonzero == 108
+    spots = {0.0: 0xF8, 2.0 ** -9: 0xF8, 0.0625: 0xF7, 0.5: 0xF2, 0.6875: 0xF0, 1.0: 0xEC,
+             2.0: 0xE1, 3.5: 0xCF, 8.0: 0x9B, 16.0: 0x3F, 20.0: 0x11, 22.0: 0x02, 24.0: 0x00,
+             896.0: 0x00}
+    for s, b in spots.items():
+        assert L.lamp_oracle_lut8(L.lamp_oracle_enc_ue5m3(s)) == b, s
+
+
+def test_exp16_rounds_to_twelve_bits():
+    for a in [0.0, -1.0, -0.5, -7.25, -20.0, -20.5, 0.75]:
+        v = L.lamp_oracle_exp16(a)
+        m, _ = math.frexp(v)
+        assert (m * 4096) == int(m * 4096)                       # 12 significant bits
+        assert abs(v - math.exp(a)) <= math.exp(a) * 2.0 ** -12
+    assert L.lamp_oracle_exp16(0.0) == 1.0
+    tiny = L.lamp_oracle_exp16(-27.0)                            # below 2^-30: quantum 2^-41
+    assert tiny / 2.0 ** -41 == round(tiny / 2.0 ** -41) and abs(tiny - math.exp(-27.0)) <= 2.0 ** -42
+    assert L.lamp_oracle_exp16(-30.0) == 0.0
+
+
+# ----------------------------------------------------------------- P11: stage 2, eq. (8)
+
+def stage2(xi, om, tau, free):
+    xi = np.ascontiguousarray(xi, np.float64); om = np.ascontiguousarray(om, np.float32)
+    return L.lamp_oracle_stage2(xi.ctypes.data_as(C.c_void_p), om.ctypes.data_as(C.c_void_p),
+                                tau, free)
+
+
+def test_stage2_hand_example_and_tie_rule():
+    xi = np.zeros((4, 32)); xi[:, 0] = [0.05, 0.3, 0.3, 0.05]
+    assert stage2(xi, np.ones(32), 0.5, 0b1111) == 0b0010
+    assert stage2(xi, np.ones(32), 1.0, 0b1111) == 0
+    assert stage2(xi, np.ones(32), 0.0, 0b1111) == 0b1111
+    assert stage2(xi, np.ones(32), 0.5, 0b1101) == 0            # 0.05+0.3+0.05 <= 0.5
+
+
+def test_stage2_is_optimal_by_brute_force():
+    rng = np.random.default_rng(1)
+    for _ in range(300):
+        free = int(rng.integers(0, 16))
+        om = rng.uniform(0.5, 3.0, 32).astype(np.float32)
+        xi = rng.uniform(0, 0.6, (4, 32)) * (rng.random((4, 32)) < 0.3)
+        for th in range(4):
+            if not (free >> th) & 1:
+                xi[th] = 0
+        tau = float(rng.choice([0.03125, 0.125, 0.5]))
+        got = stage2(xi, om, tau, free)
+        feas = [r for r in range(16) if (r & ~free) == 0 and all(
+            sum(xi[th, j] for th in range(4) if ((free & ~r) >> th) & 1)
+            <= tau * float(om[j]) * float(om[j]) for j in range(32))]
+        best = min(feas, key=lambda r: (bin(r).count("1"), r))
+        assert got == best
+
+
+# ------------------------------------------------------------------ whole-path pins
+
+def ref_attention(q, k, v, scale, causal=True, window=0):
+    B, Hq, N, D = q.shape
+    rep = Hq // k.shape[1]
+    kf = k.double().repeat_interleave(rep, 1); vf = v.double().repeat_interleave(rep, 1)
+    s = (q.double() @ kf.transpose(-1, -2)) * float(scale)
+    i = torch.arange(N)[None, :]; j = torch.arange(N)[:, None]
+    mask = torch.zeros(N, N, dtype=torch.bool)
+    if causal:
+        mask |= i > j
+    if window:
+        mask |= (j - i) >= window
+    s = s.masked_fill(mask, float("-inf"))
+    return torch.softmax(s, -1) @ vf, torch.logsumexp(s, -1), s
+
+
+def dense(res, B, Hq, N, D):
+    return (torch.from_numpy(res.out).reshape(B, Hq, N, D).double(),
+            torch.from_numpy(res.lse).reshape(B, Hq, N).double())
+
+
+@pytest.fixture(scope="module")
+def small():
+    cfg = li.CONFIGS[1]
+    q, k, v = li.make_qkv(cfg, Hq=4, Hkv=2, N=512)
+    return q, k, v, li.softmax_scale(128)
+
+
+def test_force16_matches_fp64_attention_within_16bit_bound(small):
+    q, k, v, sc = small
+    r = oracle.run_all(q, k, v, scale=sc, flags=oracle.FORCE_16BIT)
+    out, lse = dense(r, 1, 4, 512, 128)
+    o, l, s = ref_attention(q, k, v, sc)
+    # one e4m11 rounding of the logit, one 12-bit rounding of the shift, one of the
+    # exponential: relative weight error <= exp(2^-12 (|y| + |y - mu|) + 2^-12) - 1
+    smax = s.masked_fill(torch.isinf(s), 0).abs().amax(-1)
+    spread = (s.amax(-1, keepdim=True) - s).masked_fill(torch.isinf(s), 0).amax(-1)
+    rel = torch.expm1(2.0 ** -12 * (smax + spread + 1.0) + 2.0 ** -11)
+    bound = 2 * rel * v.double().abs().max()
+    assert ((out - o).abs().amax(-1) <= bound).all()
+    assert ((lse - l).abs() <= rel + 1e-6).all()
+    assert (r.flags & 0xF0).max() == 0
+
+
+def test_tau_zero_recomputes_everything_that_matters(small):
+    q, k, v, sc = small
+    r = oracle.run_all(q, k, v, scale=sc, tau=0.0)
+    out, _ = dense(r, 1, 4, 512, 128)
+    o, _, _ = ref_attention(q, k, v, sc)
+    assert (out - o).abs().max() < 5e-2
+    r8 = oracle.run_all(q, k, v, scale=sc, flags=oracle.FORCE_8BIT)
+    out8, _ = dense(r8, 1, 4, 512, 128)
+    assert (out - o).norm() < 0.2 * (out8 - o).norm()
+
+
+def test_tau_one_disables_stage_two_and_fraction_is_monotone(small):
+    q, k, v, sc = small
+    prev = None
+    for tau in [1.0, 0.5, 0.25, 0.125, 2.0 ** -4, 2.0 ** -5, 0.0]:
+        r = oracle.run_all(q, k, v, scale=sc, tau=tau)
+        if tau >= 1.0:
+            assert (r.flags & 0xF0).max() == 0            # Sec. 4.2: tau = 1 omits stage two
+        frac = (r.stats["stage1_flagged"] + r.stats["stage2_flagged"]) / r.stats["subblocks_active"]
+        if prev is not None:
+            assert frac >= prev - 0.01
+        prev = frac
+        # first tile of every unit: the first visit starts from mu = -inf, so the first
+        # active sub-block (lowest index under the tie rule) fails eq. (7)
+        assert ((r.flags[:, 0] & 1) == 1).all()
+
+
+def test_rows_sum_to_one_and_units_are_independent(small):
+    q, k, v, sc = small
+    ones = torch.ones_like(v)
+    r = oracle.run_all(q, k, ones, scale=sc)
+    assert np.abs(r.out - 1.0).max() < 1e-6
+    full = oracle.run_all(q, k, v, scale=sc)
+    pick = np.array([[0, 3, 15], [0, 0, 0], [0, 2, 7]], np.int32)
+    sub = oracle.run_units(q, k, v, pick, scale=sc)
+    for n, (b, h, g) in enumerate(pick):
+        u = h * 16 + g
+        assert np.array_equal(sub.out[n], full.out[u]) and np.array_equal(sub.flags[n], full.flags[u])
+        assert np.array_equal(sub.checks[n], full.checks[u])
+
+
+def test_force8_equals_an_independent_pure_8bit_flash_loop():
+    cfg = li.CONFIGS[1]
+    q, k, v = li.make_qkv(cfg, Hq=1, Hkv=1, N=128)
+    sc = np.float32(li.softmax_scale(128))
+    r = oracle.run_all(q, k, v, scale=sc, flags=oracle.FORCE_8BIT, dumps=True)
+    assert r.flags.max() == 0
+    e4 = lambda x: torch.tensor(np.clip(x, -448, 448), dtype=torch.float32).to(
+        torch.float8_e4m3fn).to(torch.float32).numpy()
+    grid = [L.lamp_oracle_dec_exp8(b) for b in range(0xF9)]
+    Q = q[0, 0].float().numpy(); K = k[0, 0].float().numpy(); V = v[0, 0].double().numpy()
+    qs = (Q * sc).astype(np.float32)
+    N = 128
+    for g in range(N // 32):
+        rows = slice(32 * g, 32 * g + 32)
+        mu = np.full(32, -np.inf); om = np.zeros(32); O = np.zeros((32, 128))
+        for t in range(N // 64):
+            if 64 * t > 32 * g + 31:
+                break
+            c = np.zeros((64, 32), np.float32)
+            Kt = K[64 * t:64 * t + 64]
+            for kk in range(128):      # fp64 holds the 32-bit product plus the addend exactly here
+                c = e4((Kt[:, kk:kk + 1].astype(np.float64) * qs[rows, kk][None, :].astype(np.float64)
+                        + c.astype(np.float64)).astype(np.float32))
+            valid = (64 * t + np.arange(64))[:, None] <= (32 * g + np.arange(32))[None, :]
+            ybytes = np.vectorize(lambda x: L.lamp_oracle_enc_e4m3(float(x)))(c).astype(np.uint8)
+            got = r.y8[g][:, 64 * t:64 * t + 64].T
+            assert np.array_equal(got[valid], ybytes[valid])
+            muh = np.maximum(mu, np.where(valid, c, -np.inf).max(0))
+            E = np.zeros((64, 32))
+            for i in range(64):
+                for j in range(32):
+                    if valid[i, j]:
+                        s = float(muh[j]) - float(c[i, j])
+                        m, e = math.frexp(s) if s else (0.0, 0)
+                        s4 = math.ldexp(round(m * 16) , e - 4) if s else 0.0   # 4 significant bits
+                        if s and (m * 16) % 1 == 0.5:                          # ties to even
+                            s4 = math.ldexp(2 * round(m * 8), e - 4)
+                        E[i, j] = brute_nearest_even(math.exp(-s4), grid)
+                        assert E[i, j] == L.lamp_oracle_dec_exp8(int(r.e8[g][j, 64 * t + i]))
+            lam = np.where(np.isinf(mu), 0.0, np.exp(mu - muh))
+            om = lam * om + E.sum(0)
+            O = lam[:, None] * O + E.T @ V[64 * t:64 * t + 64]
+            mu = muh
+        assert np.abs(O / om[:, None] - r.out[g]).max() < 1e-5
+        assert np.abs(mu + np.log(om) - r.lse[g]).max() < 1e-4
+
+
+def test_mass_shift_bound_eq4_on_a_single_tile():
+    """Eq. (4): the l1 distance between the computed and the exact softmax row is bounded,
+    to first order, by 2 * sum over 8-bit entries of p(1-p) times the largest relative
+    error of an input of the normalisation.  V = unit vectors makes out = probabilities."""
+    gen = torch.Generator().manual_seed(5)
+    N, D = 64, 128
+    q = (torch.randn(1, 1, N, D, generator=gen) * 0.6).to(torch.bfloat16)
+    k = (torch.randn(1, 1, N, D, generator=gen) * 0.6).to(torch.bfloat16)
+    k[0, 0, 5] += 3 * q[0, 0].float().mean(0).to(torch.bfloat16)
+    v = torch.zeros(1, 1, N, D); v[0, 0, torch.arange(N), torch.arange(N)] = 1.0
+    v = v.to(torch.bfloat16)
+    sc = li.softmax_scale(D)
+    checked = 0
+    for tau in [1.0, 0.5, 0.125]:
+        r = oracle.run_all(q, k, v, scale=sc, causal=False, tau=tau, dumps=True)
+        _, _, s = ref_attention(q, k, v, sc, causal=False)
+        p_exact = torch.softmax(s[0, 0], -1).numpy()
+        for g in range(2):
+            fl = int(r.flags[g, 0]); hi = (fl | (fl >> 4)) & 15
+            is8 = np.array([not (hi >> (i // 16)) & 1 for i in range(N)])
+            for j in range(32):
+                row = 32 * g + j
+                p = r.out[g, j, :N].astype(np.float64)
+                y = s[0, 0, row].numpy()
+                # relative error of each 8-bit input of the normalisation, measured from
+                # the oracle's own bytes: exp(shift error) times the 2^-4 rounding of the LUT
+                e8 = np.array([L.lamp_oracle_dec_exp8(int(b)) if b != 0xFF else np.nan
+                               for b in r.e8[g][j]])
+                ref = np.exp(y - y.max())
+                w = np.where(is8 & (e8 > 0), np.abs(e8 / ref - 1.0), 0.0)
+                scale_free = np.nanmedian((e8 / ref)[is8 & (e8 > 2.0 ** -20)]) if (is8 & (e8 > 2.0 ** -20)).any() else 1.0
+                w = np.where(is8 & (e8 > 0), np.abs(e8 / ref / scale_free - 1.0), 0.0)
+                winf = max(w.max(), 2.0 ** -11)
+                mass = (p_exact[row] * (1 - p_exact[row]))[is8].sum() + 2.0 ** -11
+                bound = 65 * 2.0 ** -24 + 2 * mass * winf * (1 + winf) + 2.0 ** -10
+                assert np.abs(p - p_exact[row]).sum() <= bound
+                checked += 1
+    assert checked == 192
