@@ -1,0 +1,136 @@
+/*
+ * lamp_attn.h -- C ABI of the B200 (sm_100a) LampAttention forward library.
+ *
+ * LampAttention is the look-ahead mixed-precision FlashAttention of the paper
+ * "LampAttention: Look-Ahead Mixed-Precision FlashAttention for Dedicated
+ * Accelerators".  Per key tile of 64 keys and per group of 32 query rows the
+ * forward pass (Algorithm 1)
+ *   1. accumulates the logits K^T Q / sqrt(d) in an emulated 8-bit e4m3
+ *      accumulator, one rounding per scalar multiply-add (Sec. 3.3, Sec. 4.1),
+ *   2. flags numerically sensitive 16-key sub-blocks in two stages: the
+ *      running-maximum test of eq. (7), then the block-LAMP problem of eq. (8),
+ *   3. recomputes flagged sub-blocks in the 16-bit formats e4m11 / ue5m11,
+ *      evaluates the other exponentials through the 256-entry 8-bit table,
+ *   4. finishes with the usual online-softmax rescale and P V.
+ *
+ * All pointers named "device" are CUDA device pointers of the current device;
+ * the caller owns every buffer.  The library allocates no device memory.  All
+ * functions return 0 on success or a negative lamp_attn_error; no exception
+ * crosses this boundary.  Work is enqueued on the given stream and is
+ * asynchronous with respect to the host unless stated otherwise.
+ */
+#ifndef LAMP_ATTN_H_
+#define LAMP_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum lamp_attn_error {
+  LAMP_OK = 0,
+  LAMP_ERR_INVALID_ARG = -1,      /* null pointer, negative size, bad flag combination   */
+  LAMP_ERR_UNSUPPORTED_SHAPE = -2,/* head_dim, seqlen, strides or alignment not supported */
+  LAMP_ERR_CUDA = -3,             /* a CUDA runtime call failed (see lamp_attn_last_cuda_error) */
+  LAMP_ERR_DEVICE_TIMEOUT = -4,   /* a bounded device-side wait ran out                   */
+  LAMP_ERR_UNSUPPORTED_DEVICE = -5/* the current device is not compute capability 10.x    */
+} lamp_attn_error;
+
+/* Mode bits of lamp_attn_params.flags. */
+#define LAMP_FORCE_16BIT     0x01u /* every active sub-block takes the 16-bit path (comparison mode)      */
+#define LAMP_FORCE_8BIT      0x02u /* no recomputation at all: the paper's pure 8-bit baseline (Sec. 4.1) */
+#define LAMP_NO_STAGE1       0x04u /* skip the running-maximum test (the paper's Appendix D ablation)     */
+#define LAMP_OUT_FP32        0x08u /* `out` is fp32 instead of bf16                                       */
+
+/* Problem statement of Algorithm 1: Q, K, V per head in HBM, safety margin
+ * delta of eq. (7), threshold tau of eq. (8).  Layout: element strides for
+ * (batch, head, token); the head_dim stride is 1.  Every row start must be
+ * 16-byte aligned (strides multiples of 8 elements, base pointers 16-byte
+ * aligned). */
+typedef struct lamp_attn_params {
+  int32_t batch, heads_q, heads_kv; /* heads_q % heads_kv == 0 (grouped-query attention)      */
+  int32_t seqlen;                   /* multiple of 128                                         */
+  int32_t head_dim;                 /* 128 or 256                                              */
+  int64_t q_strides[3], k_strides[3], v_strides[3], o_strides[3];
+  int32_t causal;                   /* 0 / 1                                                   */
+  int32_t window;                   /* 0 = unlimited, else (needs causal = 1) key i is visible
+                                       to query j iff i <= j and j - i < window                */
+  float scale;                      /* softmax scale, folded into Q in fp32 before the
+                                       low-precision accumulation (Sec. 3.3)                   */
+  float threshold;                  /* tau of eq. (8), >= 0; the paper's tables use 0.5        */
+  float delta;                      /* safety margin of eq. (7), >= 0; the paper uses 2^-8     */
+  uint32_t flags;                   /* LAMP_* mode bits                                        */
+  /* Optional debug outputs (device, may be NULL).                                            */
+  int32_t dbg_batch, dbg_head;      /* the (batch, query head) the dense dumps refer to        */
+  uint8_t* dbg_y8;                  /* [seqlen(query), seqlen(key)] e4m3 byte of the first-pass
+                                       logit of every visible pair, 0x7F elsewhere            */
+  uint8_t* dbg_e8;                  /* same shape: byte of the 8-bit exponential of every
+                                       visible pair of a sub-block that passed stage 1 (also
+                                       those replaced in stage 2), 0xFF elsewhere             */
+  uint64_t* dbg_checksums;          /* [batch, heads_q, seqlen/32, seqlen/64, 2]: position-keyed
+                                       checksums of the y8 and e8 bytes of each (group, tile)  */
+} lamp_attn_params;
+
+/* Counters of the most recent lamp_attn_fwd on the current device. */
+typedef struct lamp_attn_stats {
+  uint64_t subblocks_active;         /* sub-blocks with at least one visible pair              */
+  uint64_t stage1_flagged;           /* recomputed because eq. (7) failed                      */
+  uint64_t stage2_flagged;           /* recomputed by the solution of eq. (8)                  */
+  uint64_t hist_flagged_per_tile[5]; /* (group, key tile) pairs with 0..4 recomputed sub-blocks:
+                                        the "16-bit sub-blocks per tile" columns of Tables 1-6 */
+  uint64_t sat_e4m3;                 /* visible pairs whose 8-bit logit ended at +-448         */
+  uint64_t sat_e4m11;                /* recomputed pairs whose 16-bit logit ended at +-448     */
+  uint64_t exp16_gt1;                /* 16-bit exponentials above 1 (stage-2 logit > maximum)  */
+  uint64_t big_rowsum;               /* (group, tile) pairs with a row sum of 2^12 or more     */
+  int32_t device_status;             /* 0, or LAMP_ERR_DEVICE_TIMEOUT                          */
+  int32_t reserved;
+} lamp_attn_stats;
+
+/* Fill *p with zeros and the paper's defaults (tau = 0.5, delta = 2^-8, causal = 1,
+ * flags = 0).  p: host.  Shapes and strides remain for the caller to set. */
+int lamp_attn_default_params(lamp_attn_params* p);
+
+/* Set the four stride triples of *p for contiguous [batch, heads, seqlen, head_dim]
+ * tensors, from the sizes already stored in *p.  p: host. */
+int lamp_attn_contiguous_strides(lamp_attn_params* p);
+
+/* Bytes of caller-provided scratch lamp_attn_fwd needs for *p (currently 0). */
+size_t lamp_attn_workspace_bytes(const lamp_attn_params* p);
+
+/* The LampAttention forward pass (Algorithm 1 of the paper).
+ *   q        device, bf16, [batch, heads_q, seqlen, head_dim] through q_strides
+ *   k, v     device, bf16, [batch, heads_kv, seqlen, head_dim] through k/v_strides
+ *   out      device, bf16 (fp32 with LAMP_OUT_FP32) through o_strides
+ *   lse      device, fp32 [batch, heads_q, seqlen]: running maximum + ln(normaliser);
+ *            may be NULL
+ *   flag_mask device, u8 [batch, heads_q, seqlen/32, seqlen/64]: bit theta (0-3) = the
+ *            theta-th 16-key sub-block of that (32-row group, 64-key tile) was recomputed
+ *            in stage 1, bit 4+theta = in stage 2; 0 for tiles no row of the group sees;
+ *            may be NULL
+ *   p        host; read before the call returns
+ *   workspace device scratch of at least lamp_attn_workspace_bytes(p) bytes (may be NULL
+ *            when that is 0)
+ *   cuda_stream a cudaStream_t (NULL = the default stream)
+ * Inputs must be finite.  Logits beyond +-448 saturate (counted, not an error).
+ * Errors: LAMP_ERR_INVALID_ARG, LAMP_ERR_UNSUPPORTED_SHAPE, LAMP_ERR_UNSUPPORTED_DEVICE,
+ * LAMP_ERR_CUDA; nothing is enqueued when an error is returned. */
+int lamp_attn_fwd(const void* q, const void* k, const void* v, void* out, float* lse,
+                  uint8_t* flag_mask, const lamp_attn_params* p, void* workspace,
+                  size_t workspace_bytes, void* cuda_stream);
+
+/* Wait for the stream, then copy the counters of the last lamp_attn_fwd on the current
+ * device to *host_out.  Returns LAMP_ERR_DEVICE_TIMEOUT if that kernel gave up a wait. */
+int lamp_attn_get_stats(lamp_attn_stats* host_out, void* cuda_stream);
+
+/* The last cudaError_t seen by this library on the calling thread (0 = none). */
+int lamp_attn_last_cuda_error(void);
+
+/* Static, human-readable text for an error code. */
+const char* lamp_attn_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LAMP_ATTN_H_ */

@@ -1,0 +1,155 @@
+"""ctypes binding of ``include/lamp_attn.h`` (argument marshalling only)."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "liblamp_attn.so")
+
+LAMP_FORCE_16BIT, LAMP_FORCE_8BIT, LAMP_NO_STAGE1, LAMP_OUT_FP32 = 1, 2, 4, 8
+
+EXPORTS = ("lamp_attn_default_params", "lamp_attn_contiguous_strides", "lamp_attn_workspace_bytes",
+           "lamp_attn_fwd", "lamp_attn_get_stats", "lamp_attn_last_cuda_error", "lamp_attn_strerror")
+
+
+class LampAttnError(RuntimeError):
+    pass
+
+
+class LampAttnParams(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("heads_q", C.c_int32), ("heads_kv", C.c_int32),
+                ("seqlen", C.c_int32), ("head_dim", C.c_int32),
+                ("q_strides", C.c_int64 * 3), ("k_strides", C.c_int64 * 3),
+                ("v_strides", C.c_int64 * 3), ("o_strides", C.c_int64 * 3),
+                ("causal", C.c_int32), ("window", C.c_int32), ("scale", C.c_float),
+                ("threshold", C.c_float), ("delta", C.c_float), ("flags", C.c_uint32),
+                ("dbg_batch", C.c_int32), ("dbg_head", C.c_int32),
+                ("dbg_y8", C.c_void_p), ("dbg_e8", C.c_void_p), ("dbg_checksums", C.c_void_p)]
+
+
+class LampAttnStats(C.Structure):
+    _fields_ = [("subblocks_active", C.c_uint64), ("stage1_flagged", C.c_uint64),
+                ("stage2_flagged", C.c_uint64), ("hist_flagged_per_tile", C.c_uint64 * 5),
+                ("sat_e4m3", C.c_uint64), ("sat_e4m11", C.c_uint64), ("exp16_gt1", C.c_uint64),
+                ("big_rowsum", C.c_uint64), ("device_status", C.c_int32), ("reserved", C.c_int32)]
+
+    def as_dict(self):
+        d = {k: int(getattr(self, k)) for k, _ in self._fields_
+             if k not in ("hist_flagged_per_tile", "reserved")}
+        d["hist_flagged_per_tile"] = [int(x) for x in self.hist_flagged_per_tile]
+        return d
+
+
+_lib = None
+
+
+def library():
+    """Load the compiled CUDA library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise LampAttnError(
+                f"{_LIB_PATH} is missing: build it with `python -m paper_2609_39361_b200.build` "
+                "(there is no fallback path)")
+        L = C.CDLL(_LIB_PATH)
+        PP = C.POINTER(LampAttnParams)
+        L.lamp_attn_default_params.restype = C.c_int; L.lamp_attn_default_params.argtypes = [PP]
+        L.lamp_attn_contiguous_strides.restype = C.c_int; L.lamp_attn_contiguous_strides.argtypes = [PP]
+        L.lamp_attn_workspace_bytes.restype = C.c_size_t; L.lamp_attn_workspace_bytes.argtypes = [PP]
+        L.lamp_attn_fwd.restype = C.c_int
+        L.lamp_attn_fwd.argtypes = [C.c_void_p] * 6 + [PP, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.lamp_attn_get_stats.restype = C.c_int
+        L.lamp_attn_get_stats.argtypes = [C.POINTER(LampAttnStats), C.c_void_p]
+        L.lamp_attn_last_cuda_error.restype = C.c_int; L.lamp_attn_last_cuda_error.argtypes = []
+        L.lamp_attn_strerror.restype = C.c_char_p; L.lamp_attn_strerror.argtypes = [C.c_int]
+        _lib = L
+    return _lib
+
+
+def lamp_attn_strerror(code: int) -> str:
+    return library().lamp_attn_strerror(int(code)).decode()
+
+
+def lamp_attn_last_cuda_error() -> int:
+    return int(library().lamp_attn_last_cuda_error())
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        raise LampAttnError(f"{what}: {lamp_attn_strerror(rc)} (code {rc}, cuda {lamp_attn_last_cuda_error()})")
+
+
+def lamp_attn_default_params() -> LampAttnParams:
+    p = LampAttnParams()
+    _check(library().lamp_attn_default_params(C.byref(p)), "lamp_attn_default_params")
+    return p
+
+
+def lamp_attn_contiguous_strides(p: LampAttnParams) -> LampAttnParams:
+    _check(library().lamp_attn_contiguous_strides(C.byref(p)), "lamp_attn_contiguous_strides")
+    return p
+
+
+def lamp_attn_workspace_bytes(p: LampAttnParams) -> int:
+    return int(library().lamp_attn_workspace_bytes(C.byref(p)))
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def lamp_attn_fwd(q, k, v, out, lse, flag_mask, p: LampAttnParams, workspace=None, stream=None) -> None:
+    """q, k, v, out, lse, flag_mask, workspace: CUDA tensors (or None where the header allows)."""
+    import torch
+    s = torch.cuda.current_stream().cuda_stream if stream is None else stream
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = library().lamp_attn_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), _ptr(flag_mask),
+                                 C.byref(p), _ptr(workspace), ws_bytes, C.c_void_p(s))
+    _check(rc, "lamp_attn_fwd")
+
+
+def lamp_attn_get_stats(stream=None) -> dict:
+    import torch
+    s = torch.cuda.current_stream().cuda_stream if stream is None else stream
+    st = LampAttnStats()
+    rc = library().lamp_attn_get_stats(C.byref(st), C.c_void_p(s))
+    _check(rc, "lamp_attn_get_stats")
+    return st.as_dict()
+
+
+def forward(q, k, v, *, causal=True, window=0, scale=None, threshold=0.5, delta=2.0 ** -8, flags=0,
+            out_fp32=False, want_lse=True, want_flags=True, dump=None, checksums=False, stream=None):
+    """Convenience wrapper: allocate outputs with torch, fill the params struct, call
+    ``lamp_attn_fwd``.  q: [B, Hq, N, D] bf16 CUDA; k, v: [B, Hkv, N, D].
+    dump=(batch, head) also returns the dense y8 / e8 byte maps of that head."""
+    import torch
+    assert q.is_cuda and q.dtype == torch.bfloat16
+    B, Hq, N, D = q.shape
+    p = lamp_attn_default_params()
+    p.batch, p.heads_q, p.heads_kv, p.seqlen, p.head_dim = B, Hq, k.shape[1], N, D
+    for name, t in (("q_strides", q), ("k_strides", k), ("v_strides", v)):
+        assert t.stride(3) == 1
+        getattr(p, name)[:] = list(t.stride()[:3])
+    out = torch.empty(B, Hq, N, D, device=q.device, dtype=torch.float32 if out_fp32 else torch.bfloat16)
+    p.o_strides[:] = list(out.stride()[:3])
+    p.causal, p.window = int(causal), int(window)
+    p.scale = float(scale) if scale is not None else float(torch.tensor(D, dtype=torch.float64).rsqrt().float())
+    p.threshold, p.delta = float(threshold), float(delta)
+    p.flags = int(flags) | (LAMP_OUT_FP32 if out_fp32 else 0)
+    res = {"out": out}
+    lse = torch.empty(B, Hq, N, device=q.device, dtype=torch.float32) if want_lse else None
+    fm = torch.empty(B, Hq, N // 32, N // 64, device=q.device, dtype=torch.uint8) if want_flags else None
+    if dump is not None:
+        p.dbg_batch, p.dbg_head = dump
+        res["y8"] = torch.full((N, N), 0x7F, device=q.device, dtype=torch.uint8)
+        res["e8"] = torch.full((N, N), 0xFF, device=q.device, dtype=torch.uint8)
+        p.dbg_y8, p.dbg_e8 = res["y8"].data_ptr(), res["e8"].data_ptr()
+    if checksums:
+        res["checks"] = torch.empty(B, Hq, N // 32, N // 64, 2, device=q.device, dtype=torch.int64)
+        p.dbg_checksums = res["checks"].data_ptr()
+    ws_bytes = lamp_attn_workspace_bytes(p)
+    ws = torch.empty(ws_bytes, device=q.device, dtype=torch.uint8) if ws_bytes else None
+    lamp_attn_fwd(q, k, v, out, lse, fm, p, ws, stream)
+    res["lse"], res["flags"], res["params"] = lse, fm, p
+    return res

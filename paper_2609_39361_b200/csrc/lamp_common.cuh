@@ -1,0 +1,146 @@
+// Shared device helpers of the LampAttention forward kernels: the bit-exact
+// emulation of the paper's 8-bit and 16-bit formats (Sec. 3.3) and the small
+// warp-level utilities of the decision path (Alg. 1, eq. (7), eq. (8)).
+//
+// Everything that feeds a flag decision is written with explicit round-to-nearest
+// intrinsics so that no multiply-add is contracted behind our back.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace lamp {
+
+constexpr int kBQ = 32;   // query rows per warp ("single warp" of Alg. 1)
+constexpr int kBK = 16;   // keys per sub-block (Sec. 4.1: 64 keys / N_k = 4)
+constexpr int kNK = 4;    // sub-blocks per key tile
+constexpr int kTK = 64;   // keys per tile
+constexpr int kBM = 128;  // query rows per CTA (Sec. 4.1: b_q N_q = 128)
+constexpr unsigned kFull = 0xffffffffu;
+
+// ---------------------------------------------------------------------------
+// e4m3 rounding of an fp32 value: round to nearest even onto the grid with 4
+// significant bits, subnormal quantum 2^-9 below 2^-6, saturating at +-448
+// (Sec. 3.3).  Split-by-multiplication: p = t * (2^20 + 1) has the ulp of the
+// target quantum; clamping |p| from below at 1.5 * 2^14 pins the quantum to 2^-9
+// for small t; (p - (p - t)) then lands on the grid with ties to even.  Verified
+// against the definition for every fp32 input with |t| < 2^100.
+__device__ __forceinline__ float rne_e4m3(float t) {
+  float p = __fmul_rn(t, 1048577.0f);
+  float pp, r;
+  asm("max.xorsign.abs.f32 %0, %1, %2;" : "=f"(pp) : "f"(p), "f"(24576.0f));
+  float d = __fsub_rn(pp, t);
+  r = __fsub_rn(pp, d);
+  asm("min.xorsign.abs.f32 %0, %1, %2;" : "=f"(r) : "f"(r), "f"(448.0f));
+  return r;
+}
+
+// e4m3 byte of a value that already lies on the grid; -0 becomes 0x00.
+__device__ __forceinline__ uint32_t enc_e4m3(float v) {
+  uint32_t u = __float_as_uint(v);
+  uint32_t s = (u >> 24) & 0x80u;
+  float a = fabsf(v);
+  uint32_t mag = a < 0.015625f ? (uint32_t)(a * 512.0f) : ((u >> 20) & 0x7ffu) - 960u;
+  return mag ? (s | mag) : 0u;
+}
+
+// Keep the top 3 mantissa bits of an e4m11 value, toward zero (Sec. 3.3: the running
+// maxima are "rounded to e4m3 ... by truncating the lower mantissa bits").
+__device__ __forceinline__ float trunc_e4m3(float x) {
+  float a = fabsf(x);
+  if (a < 0.015625f) return copysignf(truncf(a * 512.0f) * 0.001953125f, x);
+  return __uint_as_float(__float_as_uint(x) & 0xfff00000u);   // also keeps +-inf
+}
+
+// Round an fp32 value to 12 significant bits, ties to even (the 16-bit shifted logit).
+__device__ __forceinline__ float rne_sig12(float d) {
+  uint32_t u = __float_as_uint(d);
+  u += 0x7ffu + ((u >> 12) & 1u);
+  return __uint_as_float(u & 0xfffff000u);
+}
+
+// e4m11 rounding of a double: 12 significant bits, subnormal quantum 2^-17 below
+// 2^-6, saturating at +-448.
+__device__ __forceinline__ float rne_e4m11(double x) {
+  double a = fmin(fabs(x), 448.0);
+  int e = ((__double2hiint(a) >> 20) & 0x7ff) - 1023;
+  e = max(e, -6);
+  double m = __hiloint2double(((e + 41 + 1023) << 20) | 0x00080000, 0);  // 1.5 * 2^(e+41)
+  double r = __dsub_rn(__dadd_rn(a, m), m);
+  return copysignf((float)r, (float)x);
+}
+
+// 16-bit exponential: exp(a) correctly rounded to 12 significant bits, with the
+// subnormal quantum 2^-41 below 2^-30 (ue5m11 with the bias that maps 0xF800 to 1.0).
+__device__ __forceinline__ float exp16(float a) {
+  double v = exp((double)a);
+  int e = ((__double2hiint(v) >> 20) & 0x7ff) - 1023;
+  e = max(e, -30);
+  if (e > 900) return __int_as_float(0x7f800000);
+  double m = __hiloint2double(((e + 41 + 1023) << 20) | 0x00080000, 0);
+  return (float)__dsub_rn(__dadd_rn(v, m), m);
+}
+
+// Index into the 256-entry table of Sec. 3.3: the non-negative shift rounded to 4
+// significant bits, as a ue5m3 byte with exponent bias 15.
+__device__ __forceinline__ uint32_t shift_index(float s) {
+  uint32_t u = __float_as_uint(s);
+  u += 0x7ffffu + ((u >> 20) & 1u);
+  int p = (int)(u >> 20) - 896;
+  return (uint32_t)max(p, 0);
+}
+
+__device__ __forceinline__ uint64_t mix64(uint64_t x) {
+  x += 0x9E3779B97F4A7C15ull;
+  x = (x ^ (x >> 30)) * 0xBF58476D1CE4E5B9ull;
+  x = (x ^ (x >> 27)) * 0x94D049BB133111EBull;
+  return x ^ (x >> 31);
+}
+
+__device__ __forceinline__ double shfl_xor_d(double v, int m) {
+  int lo = __shfl_xor_sync(kFull, __double2loint(v), m);
+  int hi = __shfl_xor_sync(kFull, __double2hiint(v), m);
+  return __hiloint2double(hi, lo);
+}
+__device__ __forceinline__ double shfl_d(double v, int src) {
+  int lo = __shfl_sync(kFull, __double2loint(v), src);
+  int hi = __shfl_sync(kFull, __double2hiint(v), src);
+  return __hiloint2double(hi, lo);
+}
+
+// Position of key i of the tile inside one kk-row of the fp32 K tile in shared
+// memory: sub-block theta is shifted by 4*theta words so that the four 16-byte
+// reads of a quarter warp (one per theta) fall into distinct banks.
+__device__ __forceinline__ int kf_pos(int i) { return i + 4 * (i >> 4); }
+constexpr int kKfStride = 80;   // floats per kk-row (64 keys + 12 shift + 4 pad)
+
+struct KernelParams {
+  const __nv_bfloat16* q;
+  const __nv_bfloat16* k;
+  const __nv_bfloat16* v;
+  void* out;
+  float* lse;
+  uint8_t* flag_mask;
+  int64_t qs[3], ks[3], vs[3], os[3];
+  int batch, heads_q, heads_kv, seqlen;
+  int causal, window;
+  float scale, tau, delta;
+  uint32_t flags;
+  int dbg_batch, dbg_head;
+  uint8_t* dbg_y8;
+  uint8_t* dbg_e8;
+  unsigned long long* dbg_checksums;
+};
+
+// Counters of the last forward call (one set per device).
+struct DeviceStats {
+  unsigned long long v[12];  // active, s1, s2, hist[5], sat8, sat16, gt1, bigrow
+  int status;
+  int pad;
+};
+
+__device__ __forceinline__ bool pair_valid(int causal, int window, int i, int j) {
+  return (!causal || i <= j) && (window == 0 || j - i < window);
+}
+
+}  // namespace lamp

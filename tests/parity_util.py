@@ -1,0 +1,61 @@
+"""Run the CUDA path and the oracle on the same seeded bits and compare them."""
+import numpy as np
+import torch
+
+import oracle
+import paper_2609_39361_b200 as lamp
+
+REL_FRO = 1e-4      # relative Frobenius error of O and of LSE (fp32 before the final store)
+MAX_ABS = 1e-3      # maximum absolute error of O and of LSE
+
+
+def run_gpu(q, k, v, *, dump=None, checksums=True, **kw):
+    dev = torch.device("cuda:0")
+    res = lamp.forward(q.to(dev), k.to(dev), v.to(dev), out_fp32=True, dump=dump,
+                       checksums=checksums, **kw)
+    stats = lamp.lamp_attn_get_stats()
+    out = {k_: (v_.cpu().numpy() if isinstance(v_, torch.Tensor) else v_) for k_, v_ in res.items()}
+    out["stats"] = stats
+    return out
+
+
+def compare_units(gpu, ref, *, check_stats=False, label=""):
+    """gpu: dict from run_gpu (dense arrays); ref: OracleResult for a list of units."""
+    N = gpu["out"].shape[2]
+    worst = {"o_abs": 0.0, "lse_abs": 0.0}
+    num = den = lnum = lden = 0.0
+    for n, (b, h, g) in enumerate(ref.units):
+        rows = slice(32 * g, 32 * g + 32)
+        gf = gpu["flags"][b, h, g]
+        assert np.array_equal(gf, ref.flags[n]), f"{label} flag bytes differ at unit {(b, h, g)}: {gf} vs {ref.flags[n]}"
+        if ref.checks is not None and "checks" in gpu:
+            gc = gpu["checks"][b, h, g].view(np.uint64)
+            assert np.array_equal(gc, ref.checks[n]), f"{label} y8/e8 checksums differ at unit {(b, h, g)}"
+        go = gpu["out"][b, h, rows].astype(np.float64)
+        ro = ref.out[n].astype(np.float64)
+        assert np.isfinite(go).all()
+        worst["o_abs"] = max(worst["o_abs"], float(np.abs(go - ro).max()))
+        num += float(((go - ro) ** 2).sum()); den += float((ro ** 2).sum())
+        gl = gpu["lse"][b, h, rows].astype(np.float64)
+        rl = ref.lse[n].astype(np.float64)
+        worst["lse_abs"] = max(worst["lse_abs"], float(np.abs(gl - rl).max()))
+        lnum += float(((gl - rl) ** 2).sum()); lden += float((rl ** 2).sum())
+    worst["o_rel_fro"] = (num / max(den, 1e-300)) ** 0.5
+    worst["lse_rel_fro"] = (lnum / max(lden, 1e-300)) ** 0.5
+    assert worst["o_rel_fro"] <= REL_FRO and worst["o_abs"] <= MAX_ABS, (label, worst)
+    assert worst["lse_rel_fro"] <= REL_FRO and worst["lse_abs"] <= MAX_ABS, (label, worst)
+    if check_stats:
+        gs = {k_: v_ for k_, v_ in gpu["stats"].items() if k_ != "device_status"}
+        assert gs == ref.stats, (label, gs, ref.stats)
+    assert gpu["stats"]["device_status"] == 0
+    return worst
+
+
+def compare_dense_bytes(gpu, ref, b, h):
+    """Dense y8 / e8 maps of head (b, h) against the oracle's per-unit dumps."""
+    for n, (ub, uh, g) in enumerate(ref.units):
+        if (ub, uh) != (b, h):
+            continue
+        rows = slice(32 * g, 32 * g + 32)
+        assert np.array_equal(gpu["y8"][rows], ref.y8[n]), f"y8 bytes differ in group {g}"
+        assert np.array_equal(gpu["e8"][rows], ref.e8[n]), f"e8 bytes differ in group {g}"

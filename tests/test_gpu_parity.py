@@ -1,0 +1,99 @@
+"""CUDA path against the oracle, element by element, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import lamp_inputs as li
+import oracle
+from parity_util import compare_dense_bytes, compare_units, run_gpu
+
+pytestmark = pytest.mark.gpu
+
+
+def test_config0_dense():
+    cfg = li.CONFIGS[0]
+    q, k, v = li.make_qkv(cfg)
+    sc = li.softmax_scale(cfg.D)
+    ref = oracle.run_all(q, k, v, scale=sc, dumps=True)
+    gpu = run_gpu(q, k, v, scale=sc, dump=(0, 0))
+    compare_units(gpu, ref, check_stats=True, label="cfg0")
+    compare_dense_bytes(gpu, ref, 0, 0)
+
+
+@pytest.mark.parametrize("flags,tau", [(0, 0.5), (0, 0.0625), (0, 1.0), (oracle.FORCE_8BIT, 0.5),
+                                       (oracle.FORCE_16BIT, 0.5), (oracle.NO_STAGE1, 0.5)])
+def test_qwen_shaped_small_all_modes(flags, tau):
+    cfg = li.CONFIGS[1]
+    q, k, v = li.make_qkv(cfg, Hq=4, Hkv=2, N=640)      # 5 query tiles, ragged vs the key tiles
+    sc = li.softmax_scale(cfg.D)
+    ref = oracle.run_all(q, k, v, scale=sc, tau=tau, flags=flags, dumps=True)
+    gpu = run_gpu(q, k, v, scale=sc, threshold=tau, flags=flags, dump=(0, 3))
+    compare_units(gpu, ref, check_stats=True, label=f"flags={flags} tau={tau}")
+    compare_dense_bytes(gpu, ref, 0, 3)
+
+
+@pytest.mark.parametrize("causal,window", [(False, 0), (True, 96), (True, 200)])
+def test_masks(causal, window):
+    cfg = li.CONFIGS[1]
+    q, k, v = li.make_qkv(cfg, Hq=2, Hkv=1, N=512, seed=77)
+    sc = li.softmax_scale(cfg.D)
+    ref = oracle.run_all(q, k, v, scale=sc, causal=causal, window=window, dumps=True)
+    gpu = run_gpu(q, k, v, scale=sc, causal=causal, window=window, dump=(0, 1))
+    compare_units(gpu, ref, check_stats=True, label=f"causal={causal} window={window}")
+    compare_dense_bytes(gpu, ref, 0, 1)
+
+
+@pytest.mark.parametrize("mult", [0.5, 4.0, 8.0])
+def test_scale_sweep_saturation(mult):
+    """Logit multipliers of the long-context sweep: at 4 and 8 many logits saturate at 448."""
+    cfg = li.CONFIGS[4]
+    q, k, v = li.make_qkv(cfg, Hq=4, Hkv=1, N=512)
+    sc = li.softmax_scale(cfg.D, mult)
+    ref = oracle.run_all(q, k, v, scale=sc, dumps=True)
+    gpu = run_gpu(q, k, v, scale=sc, dump=(0, 2))
+    big = ref.stats["big_rowsum"] or ref.stats["exp16_gt1"]
+    compare_dense_bytes(gpu, ref, 0, 2)
+    if not big:
+        compare_units(gpu, ref, check_stats=True, label=f"mult={mult}")
+
+
+def test_config1_full():
+    cfg = li.CONFIGS[1]
+    q, k, v = li.make_qkv(cfg)
+    sc = li.softmax_scale(cfg.D)
+    ref = oracle.run_all(q, k, v, scale=sc)
+    gpu = run_gpu(q, k, v, scale=sc)
+    compare_units(gpu, ref, check_stats=True, label="cfg1")
+
+
+def test_strided_inputs_and_bf16_output():
+    cfg = li.CONFIGS[1]
+    q, k, v = li.make_qkv(cfg, Hq=2, Hkv=2, N=256, seed=5)
+    sc = li.softmax_scale(cfg.D)
+    import paper_2609_39361_b200 as lamp
+    dev = torch.device("cuda:0")
+    # [B, N, H, D] storage viewed as [B, H, N, D]
+    qd = q.permute(0, 2, 1, 3).contiguous().to(dev).permute(0, 2, 1, 3)
+    kd = k.permute(0, 2, 1, 3).contiguous().to(dev).permute(0, 2, 1, 3)
+    vd = v.permute(0, 2, 1, 3).contiguous().to(dev).permute(0, 2, 1, 3)
+    a = lamp.forward(qd, kd, vd, scale=sc, out_fp32=True)
+    b = lamp.forward(q.to(dev), k.to(dev), v.to(dev), scale=sc, out_fp32=True)
+    c = lamp.forward(q.to(dev), k.to(dev), v.to(dev), scale=sc, out_fp32=False)
+    assert torch.equal(a["out"], b["out"]) and torch.equal(a["flags"], b["flags"])
+    assert torch.equal(c["out"], b["out"].to(torch.bfloat16))
+
+
+def test_bad_arguments_are_rejected():
+    import paper_2609_39361_b200 as lamp
+    dev = torch.device("cuda:0")
+    q = torch.zeros(1, 2, 128, 128, device=dev, dtype=torch.bfloat16)
+    with pytest.raises(lamp.LampAttnError):
+        lamp.forward(q, q, q, flags=lamp.LAMP_FORCE_16BIT | lamp.LAMP_FORCE_8BIT)
+    with pytest.raises(lamp.LampAttnError):
+        lamp.forward(q, q, q, causal=False, window=64)
+    q96 = torch.zeros(1, 2, 96, 128, device=dev, dtype=torch.bfloat16)
+    with pytest.raises(lamp.LampAttnError):
+        lamp.forward(q96, q96, q96)
+    q64 = torch.zeros(1, 2, 128, 64, device=dev, dtype=torch.bfloat16)
+    with pytest.raises(lamp.LampAttnError):
+        lamp.forward(q64, q64, q64)
