@@ -1,0 +1,307 @@
+#!/usr/bin/env python
+"""Benchmark of the LampAttention forward pass on B200.
+
+One "step" is one forward pass (the whole hot path: emulated 8-bit logits, flagging,
+16-bit recomputation, online softmax, P V) over one batch of synthetic Qwen3-8B-shaped
+input (B=4, 32 query / 8 KV heads, N=8192, head_dim 128, causal).  Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config C]
+
+With N > 1 (under torchrun) every rank runs the same workload on its own GPU: units
+(batch, head, 32-row group) are independent, so there is no data-path collective
+(weak scaling); the only communication is the timing barrier and a MAX over ranks.
+`--impl reference` times the CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import lamp_inputs as li  # noqa: E402
+
+SM_COUNT, LANES_PER_SM, SM_MAX_MHZ = 148, 128, 1965.0
+MIN_SLOTS_PER_STEP = 2.0   # one FMA plus at least one instruction for the 8-bit rounding
+
+
+def valid_pairs(cfg, window=0):
+    n = cfg.N
+    if not cfg.causal:
+        return n * n
+    if window:
+        w = min(window, n)
+        return w * (w + 1) // 2 + (n - w) * w
+    return n * (n + 1) // 2
+
+
+def flops_of(cfg, window=0):
+    return 4.0 * cfg.D * valid_pairs(cfg, window) * cfg.B * cfg.Hq
+
+
+def unit_pairs(cfg, g, window=0):
+    """Visible (query, key) pairs of the 32-row group g."""
+    tot = 0
+    for j in range(32 * g, 32 * g + 32):
+        tot += min(j + 1, window) if window else j + 1
+    return tot
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons during the timed region."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc:
+            time.sleep(0.15)
+            self.proc.terminate()
+            self.t.join(timeout=2)
+
+    def summary(self):
+        sm = [float(r[1]) for r in self.rows if len(r) >= 9 and r[1].replace(".", "").isdigit()]
+        reasons = set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) >= 9:
+                for nm, val in zip(names, r[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(nm)
+        mx = [float(r[2]) for r in self.rows if len(r) >= 9 and r[2].replace(".", "").isdigit()]
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def oracle_sample_run(cfg, q, k, v, scale, n_units, seed=11):
+    import oracle
+    units = li.sample_units(cfg, n_units, seed=seed)
+    t0 = time.perf_counter()
+    oracle.run_units(q, k, v, units, scale=scale, causal=cfg.causal, checksums=False)
+    dt = time.perf_counter() - t0
+    fl = sum(4.0 * cfg.D * unit_pairs(cfg, int(g)) for _, _, g in units)
+    return dt, fl, len(units)
+
+
+def reference_arm(args, cfg, rank):
+    """The oracle as it stands, on the host cores, on a bounded sample per step."""
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    q, k, v = li.make_qkv(cfg)
+    scale = li.softmax_scale(cfg.D)
+    cores = os.cpu_count() or 1
+    dt, fl, n = oracle_sample_run(cfg, q, k, v, scale, max(8, cores))      # calibration
+    per_unit = dt / n
+    n_units = int(max(cores, min(4096, 6.0 / max(per_unit, 1e-6))))
+    for _ in range(args.warmup and 1):
+        oracle_sample_run(cfg, q, k, v, scale, n_units)
+    tot_t = tot_f = 0.0
+    for s in range(args.steps):
+        dt, fl, n = oracle_sample_run(cfg, q, k, v, scale, n_units, seed=100 + s)
+        tot_t += dt; tot_f += fl
+    val = tot_f / tot_t / 1e12
+    sample = f"{n_units} of {cfg.B * cfg.Hq * cfg.N // 32} (b, h, 32-row group) units per step, seeded spread"
+    line = {"impl": "reference", "metric": "lamp_attention_fwd_tflops", "value": val, "unit": "TFLOP/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": 1e3 * tot_t / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "e4m3-emulated/f32", "data": "synthetic",
+            "config": workload_config(cfg),
+            "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def workload_config(cfg):
+    return {"workload": f"config {cfg.index}: {cfg.name} prefill, B={cfg.B}, Hq={cfg.Hq}, Hkv={cfg.Hkv}, "
+                        f"N={cfg.N}, head_dim={cfg.D}, causal, tau=0.5, delta=2^-8",
+            "l2": "inputs (Q+K+V+O = %.0f MB) larger than the 126 MB L2" %
+                  ((2 * cfg.B * cfg.Hq + 2 * cfg.B * cfg.Hkv) * cfg.N * cfg.D * 2 / 1e6)}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    cfg = li.CONFIGS[args.config]
+
+    if args.impl == "reference":
+        reference_arm(args, cfg, rank)
+        return
+
+    import paper_2609_39361_b200 as lamp
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    scale = li.softmax_scale(cfg.D)
+    q, k, v = li.make_qkv(cfg)
+    hq, hk, hv = q.pin_memory(), k.pin_memory(), v.pin_memory()
+    dq, dk, dv = hq.to(dev), hk.to(dev), hv.to(dev)
+    B, Hq, N, D = q.shape
+    out = torch.empty(B, Hq, N, D, device=dev, dtype=torch.bfloat16)
+    lse = torch.empty(B, Hq, N, device=dev, dtype=torch.float32)
+    fm = torch.empty(B, Hq, N // 32, N // 64, device=dev, dtype=torch.uint8)
+    p = lamp.lamp_attn_default_params()
+    p.batch, p.heads_q, p.heads_kv, p.seqlen, p.head_dim = B, Hq, k.shape[1], N, D
+    lamp.lamp_attn_contiguous_strides(p)
+    p.causal, p.scale = 1, scale
+    fl = flops_of(cfg)
+
+    def step():
+        lamp.lamp_attn_fwd(dq, dk, dv, out, lse, fm, p)
+
+    # ---- device-resident timing ---------------------------------------------------------
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    with ClockSampler(local_rank) as clk:
+        barrier()
+        ev[0].record()
+        for i in range(args.steps):
+            step()
+            ev[i + 1].record()
+        barrier()
+    per = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
+    total_ms = ev[0].elapsed_time(ev[-1])
+    stats = lamp.lamp_attn_get_stats()
+    t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * fl / (ms_per_step * 1e-3) / 1e12
+
+    # ---- end to end: pinned host inputs in, result out, every step -------------------------
+    ho = torch.empty(B, Hq, N, D, dtype=torch.bfloat16).pin_memory()
+    hl = torch.empty(B, Hq, N, dtype=torch.float32).pin_memory()
+    hf = torch.empty(B, Hq, N // 32, N // 64, dtype=torch.uint8).pin_memory()
+
+    def e2e_step():
+        dq.copy_(hq, non_blocking=True); dk.copy_(hk, non_blocking=True); dv.copy_(hv, non_blocking=True)
+        step()
+        ho.copy_(out, non_blocking=True); hl.copy_(lse, non_blocking=True); hf.copy_(fm, non_blocking=True)
+
+    e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    t = torch.tensor([e0.elapsed_time(e1)], device=dev, dtype=torch.float64)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_ms = float(t.item()) / args.steps
+    h2d = sum(x.numel() * x.element_size() for x in (hq, hk, hv))
+    d2h = sum(x.numel() * x.element_size() for x in (ho, hl, hf))
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the one kernel: plain-ALU issue bound ---------------------------------
+    # Each of the D * pairs emulated accumulate steps needs an fp32 FMA and at least one more
+    # instruction to round to e4m3 (no B200 instruction does both): >= 2 issue slots per step,
+    # on 148 SMs x 128 lanes at the maximum SM clock.  In the metric's FLOP convention
+    # (4 * D * pairs) that bound is 2 * 148 * 128 * 1.965 GHz = 74.4 TFLOP/s.
+    kern_ms = statistics.mean(per)
+    achieved = fl / (kern_ms * 1e-3) / 1e12
+    peak = 4.0 / MIN_SLOTS_PER_STEP * SM_COUNT * LANES_PER_SM * SM_MAX_MHZ * 1e6 / 1e12
+    traffic = None
+    tfile = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    if os.path.exists(tfile):
+        traffic = json.load(open(tfile)).get(f"config{cfg.index}_bytes_per_launch")
+    roofline = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                "frac": achieved / peak, "traffic": traffic,
+                "note": "peak = issue-slot bound of the emulated e4m3 accumulation at 2 slots/step, "
+                        "148 SMs x 128 lanes x 1965 MHz (derived, not a measured peak)"}
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        import oracle
+        oracle.build()
+        cores = os.cpu_count() or 1
+        dt, f1, n = oracle_sample_run(cfg, q, k, v, scale, max(8, cores))
+        n_units = int(max(cores, min(4096, 15.0 / max(dt / n, 1e-6))))
+        dt, f1, n = oracle_sample_run(cfg, q, k, v, scale, n_units, seed=12)
+        cpu = {"value": f1 / dt / 1e12, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
+               "sample": f"{n} of {B * Hq * N // 32} (b, h, 32-row group) units, seeded spread, {dt:.1f} s"}
+
+    act = max(stats["subblocks_active"], 1)
+    hist = stats["hist_flagged_per_tile"]
+    ht = max(sum(hist), 1)
+    line = {"metric": "lamp_attention_fwd_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "e4m3-emulated/f32", "data": "synthetic", "config": workload_config(cfg),
+            "clocks": clk.summary(),
+            "e2e": {"value": world * fl / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+            "gpu_launches": args.steps,
+            "roofline": roofline, "cpu_baseline": cpu,
+            "recomputed_subblock_pct": 100.0 * (stats["stage1_flagged"] + stats["stage2_flagged"]) / act,
+            "stage1_pct": 100.0 * stats["stage1_flagged"] / act,
+            "stage2_pct": 100.0 * stats["stage2_flagged"] / act,
+            "tiles_with_0_1_2plus_recomputed_pct": [100.0 * hist[0] / ht, 100.0 * hist[1] / ht,
+                                                    100.0 * sum(hist[2:]) / ht],
+            "saturated_logits": {"e4m3": stats["sat_e4m3"], "e4m11": stats["sat_e4m11"]}}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

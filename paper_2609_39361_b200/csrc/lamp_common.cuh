@@ -19,20 +19,24 @@ constexpr int kBM = 128;  // query rows per CTA (Sec. 4.1: b_q N_q = 128)
 constexpr unsigned kFull = 0xffffffffu;
 
 // ---------------------------------------------------------------------------
-// e4m3 rounding of an fp32 value: round to nearest even onto the grid with 4
+// e4m3 rounding of two fp32 values: round to nearest even onto the grid with 4
 // significant bits, subnormal quantum 2^-9 below 2^-6, saturating at +-448
-// (Sec. 3.3).  Split-by-multiplication: p = t * (2^20 + 1) has the ulp of the
-// target quantum; clamping |p| from below at 1.5 * 2^14 pins the quantum to 2^-9
-// for small t; (p - (p - t)) then lands on the grid with ties to even.  Verified
-// against the definition for every fp32 input with |t| < 2^100.
+// (Sec. 3.3).  B200 has no arithmetic in this format, but its conversion unit rounds
+// to it exactly: f32 pair -> e4m3 pair (nearest even, saturating), then back through
+// f16 (every e4m3 value is an f16 value).  Checked against the definition for every
+// fp32 input with |t| < 2^100.
+__device__ __forceinline__ void rne_e4m3_x2(float& a, float& b) {
+  unsigned short pk;
+  unsigned int h2;
+  asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(pk) : "f"(b), "f"(a));
+  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"(pk));
+  asm("{.reg .f16 lo, hi; mov.b32 {lo, hi}, %2; cvt.f32.f16 %0, lo; cvt.f32.f16 %1, hi;}"
+      : "=f"(a), "=f"(b) : "r"(h2));
+}
 __device__ __forceinline__ float rne_e4m3(float t) {
-  float p = __fmul_rn(t, 1048577.0f);
-  float pp, r;
-  asm("max.xorsign.abs.f32 %0, %1, %2;" : "=f"(pp) : "f"(p), "f"(24576.0f));
-  float d = __fsub_rn(pp, t);
-  r = __fsub_rn(pp, d);
-  asm("min.xorsign.abs.f32 %0, %1, %2;" : "=f"(r) : "f"(r), "f"(448.0f));
-  return r;
+  float z = 0.0f;
+  rne_e4m3_x2(t, z);
+  return t;
 }
 
 // e4m3 byte of a value that already lies on the grid; -0 becomes 0x00.

@@ -49,7 +49,13 @@ __device__ __forceinline__ void chain8(const float* __restrict__ qs, int qstride
 #pragma unroll
     for (int a = 0; a < 4; ++a)
 #pragma unroll
-      for (int b = 0; b < 16; ++b) acc[a][b] = rne_e4m3(__fmaf_rn(kv[b], q4[a], acc[a][b]));
+      for (int b = 0; b < 16; b += 2) {
+        float t0 = __fmaf_rn(kv[b], q4[a], acc[a][b]);
+        float t1 = __fmaf_rn(kv[b + 1], q4[a], acc[a][b + 1]);
+        rne_e4m3_x2(t0, t1);
+        acc[a][b] = t0;
+        acc[a][b + 1] = t1;
+      }
   }
 }
 
