@@ -8,7 +8,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(_HERE)
 SRC = os.path.join(_HERE, "csrc", "lamp_attn.cu")
 LIB = os.path.join(_HERE, "liblamp_attn.so")
-DEPS = [SRC] + [os.path.join(_HERE, "csrc", f) for f in ("lamp_common.cuh", "lamp_tile.cuh")] + [
+DEPS = [SRC] + [os.path.join(_HERE, "csrc", f) for f in ("lamp_common.cuh", "lamp_fwd_sm100.cuh", "sm100_ptx.cuh")] + [
     os.path.join(ROOT, "include", "lamp_attn.h")]
 
 NVCC_FLAGS = [

@@ -5,190 +5,18 @@
 #include <string.h>
 
 #include "lamp_common.cuh"
-#include "lamp_tile.cuh"
+#include "lamp_fwd_sm100.cuh"
 
 namespace lamp {
 
 __device__ DeviceStats g_stats;
-__constant__ uint32_t c_lut8[256];   // fp32 bits of the 8-bit exponential | its byte
+__device__ uint32_t g_lut8[256];   // fp32 bits of the 8-bit exponential | its byte
 
-// ---------------------------------------------------------------------------------------
-// Reference-structure kernel: CUDA cores only.  One CTA = 128 query rows of one (b, h),
-// four warps, one group of 32 rows each; key tiles visited in ascending order (the flags
-// depend on the history of the running maxima, so the key dimension is never split).
-template <int D, bool DUMP>
-__global__ void __launch_bounds__(128, 1) lamp_fwd_simt(const __grid_constant__ KernelParams P) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  float* qsT = reinterpret_cast<float*>(smem_raw);                    // [D][128] q * scale
-  float* kf = qsT + D * kBM;                                          // [D][kKfStride]
-  __nv_bfloat16* vs = reinterpret_cast<__nv_bfloat16*>(kf + D * kKfStride);  // [64][D]
-  float* es_all = reinterpret_cast<float*>(vs + kTK * D);             // [4][64][32]
-  float* os = es_all + 4 * kTK * kBQ;                                 // [128][D]
-  float* rowbuf = os + kBM * D;                                       // [128]
-  uint32_t* lut = reinterpret_cast<uint32_t*>(rowbuf + kBM);          // [256]
-
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int qa = lane >> 2, th_own = lane & 3;
-  const int ntq = P.seqlen / kBM;
-  const int qt = ntq - 1 - blockIdx.x;            // long (late) query tiles first
-  const int h = blockIdx.y, b = blockIdx.z;
-  const int hk = h / (P.heads_q / P.heads_kv);
-  const int m0 = qt * kBM;
-  const int j0 = m0 + warp * kBQ;
-
-  const __nv_bfloat16* qg = P.q + b * P.qs[0] + h * P.qs[1] + (int64_t)m0 * P.qs[2];
-  const __nv_bfloat16* kg = P.k + b * P.ks[0] + hk * P.ks[1];
-  const __nv_bfloat16* vg = P.v + b * P.vs[0] + hk * P.vs[1];
-
-  for (int i = tid; i < 256; i += 128) lut[i] = c_lut8[i];
-  for (int c = tid; c < kBM * D / 8; c += 128) {
-    const int row = c / (D / 8), k0 = (c % (D / 8)) * 8;
-    const uint4 raw = *reinterpret_cast<const uint4*>(qg + (int64_t)row * P.qs[2] + k0);
-#pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      const uint32_t w = (&raw.x)[e >> 1];
-      const float f = __uint_as_float((e & 1) ? (w & 0xffff0000u) : (w << 16));
-      qsT[(k0 + e) * kBM + row] = __fmul_rn(f, P.scale);
-    }
-  }
-  for (int c = tid; c < kBM * D; c += 128) os[c] = 0.0f;
-
-  RowState st;
-#pragma unroll
-  for (int a = 0; a < 4; ++a) { st.mu[a] = -INFINITY; st.om[a] = 0.0f; }
-  WarpCounters wc;
-  memset(&wc, 0, sizeof(wc));
-
-  int t_begin = 0, t_end = P.seqlen / kTK;
-  if (P.causal) t_end = min(t_end, (m0 + kBM - 1) / kTK + 1);
-  if (P.window > 0) t_begin = max(0, m0 - P.window + 1) / kTK;
-  const int ntk = P.seqlen / kTK;
-  const bool dump_rows = DUMP && b == P.dbg_batch && h == P.dbg_head;
-  float* es = es_all + warp * kTK * kBQ;
-
-  for (int t = t_begin; t < t_end; ++t) {
-    const int i0 = t * kTK;
-    __syncthreads();   // previous tile fully consumed
-    for (int c = tid; c < kTK * D / 8; c += 128) {
-      const int key = c / (D / 8), k0 = (c % (D / 8)) * 8;
-      const uint4 raw = *reinterpret_cast<const uint4*>(kg + (int64_t)(i0 + key) * P.ks[2] + k0);
-      const uint4 rawv = *reinterpret_cast<const uint4*>(vg + (int64_t)(i0 + key) * P.vs[2] + k0);
-      *reinterpret_cast<uint4*>(vs + key * D + k0) = rawv;
-#pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        const uint32_t w = (&raw.x)[e >> 1];
-        kf[(k0 + e) * kKfStride + kf_pos(key)] =
-            __uint_as_float((e & 1) ? (w & 0xffff0000u) : (w << 16));
-      }
-    }
-    __syncthreads();
-
-    TileGeom g;
-    g.i0 = i0; g.j0 = j0; g.causal = P.causal; g.window = P.window;
-    const bool any = (!P.causal || i0 <= j0 + 31) && (P.window == 0 || j0 - (i0 + 63) < P.window);
-    g.full = (!P.causal || i0 + 63 <= j0) && (P.window == 0 || (j0 + 31) - i0 < P.window);
-    float lam[4] = {1.0f, 1.0f, 1.0f, 1.0f};
-    uint32_t flag = 0;
-    unsigned long long cks[2] = {0ull, 0ull};
-    if (any) {
-      const int dump0 = dump_rows ? j0 : -1;
-      const __nv_bfloat16* qrow = qg + (int64_t)(warp * kBQ + 4 * qa) * P.qs[2];
-      if (g.full)
-        flag = lamp_tile<D, true, DUMP>(P, g, qsT + warp * kBQ + 4 * qa, kBM, kf, qrow, lut, es,
-                                        st, lam, wc, cks, dump0);
-      else
-        flag = lamp_tile<D, false, DUMP>(P, g, qsT + warp * kBQ + 4 * qa, kBM, kf, qrow, lut, es,
-                                         st, lam, wc, cks, dump0);
-    }
-    const int64_t gt = (((int64_t)b * P.heads_q + h) * (P.seqlen / kBQ) + (j0 / kBQ)) * ntk + t;
-    if (lane == 0 && P.flag_mask) P.flag_mask[gt] = (uint8_t)flag;
-    if (DUMP && P.dbg_checksums) {
-#pragma unroll
-      for (int s = 16; s > 0; s >>= 1) {
-        cks[0] += __shfl_xor_sync(kFull, cks[0], s);
-        cks[1] += __shfl_xor_sync(kFull, cks[1], s);
-      }
-      if (lane == 0) { P.dbg_checksums[2 * gt] = cks[0]; P.dbg_checksums[2 * gt + 1] = cks[1]; }
-    }
-    if (!any) continue;   // warp-uniform; the __syncthreads above are outside this branch
-
-    // O <- diag(lambda) O + E^T V on the CUDA cores (fp32): lane = 4 output columns
-    if (th_own == 0) {
-#pragma unroll
-      for (int a = 0; a < 4; ++a) rowbuf[warp * kBQ + 4 * qa + a] = lam[a];
-    }
-    __syncwarp();
-    for (int jq = 0; jq < kBQ; jq += 4) {
-      float o[4][D / 32];
-#pragma unroll
-      for (int a = 0; a < 4; ++a)
-#pragma unroll
-        for (int c = 0; c < D / 32; ++c)
-          o[a][c] = rowbuf[warp * kBQ + jq + a] * os[(warp * kBQ + jq + a) * D + lane + 32 * c];
-      for (int i = 0; i < kTK; ++i) {
-        const float4 e4 = *reinterpret_cast<const float4*>(es + i * kBQ + jq);
-        if (e4.x == 0.0f && e4.y == 0.0f && e4.z == 0.0f && e4.w == 0.0f) continue;
-#pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-          const float vv = __bfloat162float(vs[i * D + lane + 32 * c]);
-          o[0][c] = fmaf(e4.x, vv, o[0][c]);
-          o[1][c] = fmaf(e4.y, vv, o[1][c]);
-          o[2][c] = fmaf(e4.z, vv, o[2][c]);
-          o[3][c] = fmaf(e4.w, vv, o[3][c]);
-        }
-      }
-#pragma unroll
-      for (int a = 0; a < 4; ++a)
-#pragma unroll
-        for (int c = 0; c < D / 32; ++c) os[(warp * kBQ + jq + a) * D + lane + 32 * c] = o[a][c];
-    }
-    __syncwarp();
-  }
-
-  // ---- epilogue: O / omega, lse = mu + ln(omega) ------------------------------------------
-  if (th_own == 0) {
-#pragma unroll
-    for (int a = 0; a < 4; ++a) {
-      rowbuf[warp * kBQ + 4 * qa + a] = st.om[a];
-      if (P.lse)
-        P.lse[((int64_t)b * P.heads_q + h) * P.seqlen + j0 + 4 * qa + a] =
-            (float)((double)st.mu[a] + log((double)st.om[a]));
-    }
-  }
-  __syncwarp();
-  for (int j = 0; j < kBQ; ++j) {
-    const float den = rowbuf[warp * kBQ + j];
-    const int64_t orow = b * P.os[0] + h * P.os[1] + (int64_t)(j0 + j) * P.os[2];
-#pragma unroll
-    for (int c = 0; c < D / 32; ++c) {
-      const float val = os[(warp * kBQ + j) * D + lane + 32 * c] / den;
-      if (P.flags & LAMP_OUT_FP32) reinterpret_cast<float*>(P.out)[orow + lane + 32 * c] = val;
-      else reinterpret_cast<__nv_bfloat16*>(P.out)[orow + lane + 32 * c] = __float2bfloat16(val);
-    }
-  }
-
-  // ---- counters --------------------------------------------------------------------------
-  const unsigned sat8 = __reduce_add_sync(kFull, wc.sat8);
-  const unsigned sat16 = __reduce_add_sync(kFull, wc.sat16);
-  const unsigned gt1 = __reduce_add_sync(kFull, wc.gt1);
-  if (lane == 0) {
-    atomicAdd(&g_stats.v[0], wc.active);
-    atomicAdd(&g_stats.v[1], wc.s1);
-    atomicAdd(&g_stats.v[2], wc.s2);
-#pragma unroll
-    for (int i = 0; i < 5; ++i) atomicAdd(&g_stats.v[3 + i], wc.hist[i]);
-    atomicAdd(&g_stats.v[8], (unsigned long long)sat8);
-    atomicAdd(&g_stats.v[9], (unsigned long long)sat16);
-    atomicAdd(&g_stats.v[10], (unsigned long long)gt1);
-    atomicAdd(&g_stats.v[11], wc.bigrow);
-  }
-}
-
-template <int D>
-constexpr size_t simt_smem_bytes() {
-  return sizeof(float) * (D * kBM + D * kKfStride + 4 * kTK * kBQ + kBM * D + kBM) +
-         sizeof(__nv_bfloat16) * kTK * D + 256 * sizeof(uint32_t);
-}
+typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                      const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                      CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                      CUtensorMapFloatOOBfill);
+static TensorMapEncodeFn g_encode = nullptr;
 
 // ---------------------------------------------------------------------------------------
 // Host side: the exponential table, argument checks, launch.
@@ -216,6 +44,8 @@ static uint32_t exp8_entry(double s) {
   memcpy(&bits, &rf, 4);
   return (bits & 0xffffff00u) | byte;
 }
+
+constexpr int kSmemLaunch128 = Smem<128>::kBytes + 1024;   // + slack to align the base to 1024 B
 
 static thread_local int t_last_cuda = 0;
 static int cuda_fail(cudaError_t e) {
@@ -245,16 +75,38 @@ static int ensure_device(int* dev_out) {
     const double s = E ? ldexp(1.0 + M / 8.0, E - 15) : ldexp(M / 8.0, -14);
     lut[p] = exp8_entry(s);
   }
-  e = cudaMemcpyToSymbol(c_lut8, lut, sizeof(lut));
+  e = cudaMemcpyToSymbol(g_lut8, lut, sizeof(lut));
   if (e != cudaSuccess) return cuda_fail(e);
-  e = cudaFuncSetAttribute(lamp_fwd_simt<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           (int)simt_smem_bytes<128>());
+  if (!g_encode) {
+    cudaDriverEntryPointQueryResult qr;
+    void* fn = nullptr;
+    e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qr);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (!fn || qr != cudaDriverEntryPointSuccess) return cuda_fail(cudaErrorNotSupported);
+    g_encode = (TensorMapEncodeFn)fn;
+  }
+  e = cudaFuncSetAttribute(lamp_fwd_sm100<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLaunch128);
   if (e != cudaSuccess) return cuda_fail(e);
-  e = cudaFuncSetAttribute(lamp_fwd_simt<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           (int)simt_smem_bytes<128>());
+  e = cudaFuncSetAttribute(lamp_fwd_sm100<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLaunch128);
   if (e != cudaSuccess) return cuda_fail(e);
   if (dev < 64) g_init.ready[dev] = true;
   return LAMP_OK;
+}
+
+// K / V as a 4-D tensor (head_dim, token, head, batch) with boxes of 64 channels x 64 tokens,
+// 128-byte swizzle: the layout tcgen05.mma reads and the converter warps undo.
+static int make_kv_map(CUtensorMap* m, const void* base, const int64_t* strides, int D, int N, int H, int B) {
+  cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)N, (cuuint64_t)H, (cuuint64_t)B};
+  cuuint64_t st[3] = {(cuuint64_t)strides[2] * 2, (cuuint64_t)strides[1] * 2, (cuuint64_t)strides[0] * 2};
+  // a size-1 dimension may come with stride 0; the encoder wants a positive multiple of 16
+  for (int i = 0; i < 3; ++i)
+    if (st[i] == 0) st[i] = 16;
+  cuuint32_t box[4] = {64, 64, 1, 1};
+  cuuint32_t es[4] = {1, 1, 1, 1};
+  CUresult r = g_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, st, box, es,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? LAMP_OK : LAMP_ERR_UNSUPPORTED_SHAPE;
 }
 
 static bool strides_ok(const int64_t* s, int D) {
@@ -358,11 +210,22 @@ int lamp_attn_fwd(const void* q, const void* k, const void* v, void* out, float*
     e = cudaMemsetAsync(p->dbg_checksums, 0, ngt * 16, stream);
     if (e != cudaSuccess) return cuda_fail(e);
   }
+  void* lut_ptr = nullptr;
+  e = cudaGetSymbolAddress(&lut_ptr, g_lut8);
+  if (e != cudaSuccess) return cuda_fail(e);
+  CUtensorMap kmap, vmap;
+  rc = make_kv_map(&kmap, k, p->k_strides, p->head_dim, p->seqlen, p->heads_kv, p->batch);
+  if (rc) return rc;
+  rc = make_kv_map(&vmap, v, p->v_strides, p->head_dim, p->seqlen, p->heads_kv, p->batch);
+  if (rc) return rc;
   const bool dump = p->dbg_y8 || p->dbg_e8 || p->dbg_checksums;
-  dim3 grid(p->seqlen / kBM, p->heads_q, p->batch), block(128);
-  const size_t smem = simt_smem_bytes<128>();
-  if (dump) lamp_fwd_simt<128, true><<<grid, block, smem, stream>>>(P);
-  else lamp_fwd_simt<128, false><<<grid, block, smem, stream>>>(P);
+  dim3 grid(p->seqlen / kBM, p->heads_q, p->batch), block(kThreads);
+  if (dump)
+    lamp_fwd_sm100<128, true><<<grid, block, kSmemLaunch128, stream>>>(P, kmap, vmap, (const uint32_t*)lut_ptr,
+                                                                       (DeviceStats*)stats_ptr);
+  else
+    lamp_fwd_sm100<128, false><<<grid, block, kSmemLaunch128, stream>>>(P, kmap, vmap, (const uint32_t*)lut_ptr,
+                                                                        (DeviceStats*)stats_ptr);
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
   return LAMP_OK;

@@ -1,0 +1,768 @@
+// The sm_100a LampAttention forward kernel (Algorithm 1 of the paper).
+//
+// One CTA = 128 query rows of one (batch, query head); key tiles of 64 keys are visited
+// in ascending order (the flags depend on the history of the running maxima, so the key
+// dimension is never split across CTAs).  Seven warps, specialised:
+//
+//   warps 0-3  compute: warp w owns the group of 32 rows 32w..32w+31 (and TMEM lanes
+//              32w..32w+31).  Per tile: emulated e4m3 logits on the CUDA cores, stage 1,
+//              exponentials, stage 2, recomputation, rescale of O, P tile to shared memory.
+//   warps 4-5  convert the bf16 K tile that TMA delivered into the fp32, key-contiguous
+//              layout the chain reads (double buffered, one tile ahead of the compute warps).
+//   warp  6    lane 0 issues the TMA loads of K and V and the tcgen05 MMAs O += P V
+//              (bf16 x bf16 -> fp32 in TMEM; 16-bit exponentials enter as bf16 hi + lo).
+//
+// All hand-offs are mbarriers with bounded waits: a wait that runs out records
+// LAMP_ERR_DEVICE_TIMEOUT and lets the kernel finish instead of hanging the device.
+#pragma once
+#include "lamp_common.cuh"
+#include "sm100_ptx.cuh"
+
+namespace lamp {
+
+constexpr int kThreads = 224;
+constexpr int kCtrlWarp = 6;
+constexpr int kConvWarps = 2;
+constexpr int kTimeoutCode = -4;   // LAMP_ERR_DEVICE_TIMEOUT
+
+template <int D>
+struct Smem {
+  static constexpr int kQs = 0;                                   // [D][128] fp32
+  static constexpr int kKf = kQs + D * kBM * 4;                   // 2 x [D][kKfStride] fp32
+  static constexpr int kKbf = kKf + 2 * D * kKfStride * 4;        // D/64 boxes [64 keys][64] bf16, SW128
+  static constexpr int kV = kKbf + kTK * D * 2;                   // D/64 boxes [64 keys][64] bf16, SW128
+  static constexpr int kPhi = kV + kTK * D * 2;                   // [128][64] bf16, SW128 K-major
+  static constexpr int kPlo = kPhi + kBM * kTK * 2;
+  static constexpr int kLut = kPlo + kBM * kTK * 2;               // 256 x u32
+  static constexpr int kBar = kLut + 1024;                        // mbarriers
+  static constexpr int kMisc = kBar + 128;                        // tmem slot, lo masks
+  static constexpr int kBytes = kMisc + 64;
+  static_assert(kKbf % 1024 == 0 && kV % 1024 == 0 && kPhi % 1024 == 0 && kPlo % 1024 == 0, "swizzle atoms");
+};
+
+enum Bar { kKbfFull = 0, kKbfEmpty, kKfFull0, kKfFull1, kKfEmpty0, kKfEmpty1, kVFull, kPReady, kPvDone, kNumBars };
+
+struct TileGeom {
+  int i0, j0, causal, window;
+};
+template <bool FULL>
+__device__ __forceinline__ bool vis(const TileGeom& g, int i, int j) {
+  return FULL || pair_valid(g.causal, g.window, g.i0 + i, g.j0 + j);
+}
+
+__device__ __forceinline__ void fma_x2(float& d0, float& d1, float a0, float a1, uint64_t bb, float c0, float c1) {
+  asm("{.reg .b64 ra, rc, rd; mov.b64 ra, {%2, %3}; mov.b64 rc, {%5, %6};"
+      " fma.rn.f32x2 rd, ra, %4, rc; mov.b64 {%0, %1}, rd;}"
+      : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "l"(bb), "f"(c0), "f"(c1));
+}
+
+// First pass: Y8[i][j] = chain over kk of c <- RNE_e4m3(fma(k, q*scale, c)), c0 = +0
+// (Alg. 1 "accumulate Y in low precision"; Sec. 4.1 round(c + a*b)).  Operands of the next
+// kk are fetched while the current one is processed; FMAs are issued in packed pairs.
+template <int D>
+__device__ __forceinline__ void chain8(const float* __restrict__ qs, const float* __restrict__ kf,
+                                       float (&acc)[4][16]) {
+#pragma unroll
+  for (int a = 0; a < 4; ++a)
+#pragma unroll
+    for (int b = 0; b < 16; ++b) acc[a][b] = 0.0f;
+  float4 qn = *reinterpret_cast<const float4*>(qs);
+  float4 kn[4];
+#pragma unroll
+  for (int c = 0; c < 4; ++c) kn[c] = *reinterpret_cast<const float4*>(kf + 4 * c);
+#pragma unroll 2
+  for (int kk = 0; kk < D; ++kk) {
+    const float q4[4] = {qn.x, qn.y, qn.z, qn.w};
+    float kv[16];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) { kv[4 * c] = kn[c].x; kv[4 * c + 1] = kn[c].y; kv[4 * c + 2] = kn[c].z; kv[4 * c + 3] = kn[c].w; }
+    const int nx = (kk + 1) & (D - 1);
+    qn = *reinterpret_cast<const float4*>(qs + nx * kBM);
+#pragma unroll
+    for (int c = 0; c < 4; ++c) kn[c] = *reinterpret_cast<const float4*>(kf + nx * kKfStride + 4 * c);
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+      uint64_t qq;
+      asm("mov.b64 %0, {%1, %1};" : "=l"(qq) : "f"(q4[a]));
+#pragma unroll
+      for (int b = 0; b < 16; b += 2) {
+        float t0, t1;
+        fma_x2(t0, t1, kv[b], kv[b + 1], qq, acc[a][b], acc[a][b + 1]);
+        rne_e4m3_x2(t0, t1);
+        acc[a][b] = t0;
+        acc[a][b + 1] = t1;
+      }
+    }
+  }
+}
+
+// 16-bit logits of sub-block th for this lane's (quad x 4 keys): a sequential fp64 fma
+// chain over kk, scaled, rounded once to e4m11.
+template <int D>
+__device__ __forceinline__ void dot16(const float* __restrict__ kf, const __nv_bfloat16* qrow, int64_t qstride,
+                                      int th, int tp, double scale_d, float (&y)[4][4]) {
+  double acc[4][4];
+#pragma unroll
+  for (int a = 0; a < 4; ++a)
+#pragma unroll
+    for (int b = 0; b < 4; ++b) acc[a][b] = 0.0;
+  const float* kcol = kf + kf_pos(16 * th + 4 * tp);
+  for (int k0 = 0; k0 < D; k0 += 8) {
+    uint4 qraw[4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a) qraw[a] = *reinterpret_cast<const uint4*>(qrow + a * qstride + k0);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const float4 kq = *reinterpret_cast<const float4*>(kcol + (k0 + e) * kKfStride);
+      const double kd[4] = {(double)kq.x, (double)kq.y, (double)kq.z, (double)kq.w};
+#pragma unroll
+      for (int a = 0; a < 4; ++a) {
+        const uint32_t w = (&qraw[a].x)[e >> 1];
+        const double qd = (double)__uint_as_float((e & 1) ? (w & 0xffff0000u) : (w << 16));
+#pragma unroll
+        for (int b = 0; b < 4; ++b) acc[a][b] = fma(kd[b], qd, acc[a][b]);
+      }
+    }
+  }
+#pragma unroll
+  for (int a = 0; a < 4; ++a)
+#pragma unroll
+    for (int b = 0; b < 4; ++b) y[a][b] = rne_e4m11(__dmul_rn(scale_d, acc[a][b]));
+}
+
+// active, s1, s2, hist, bigrow are warp-uniform; sat8, sat16, gt1 are per-lane partial counts.
+struct WarpCounters {
+  unsigned long long active, s1, s2, hist[5], bigrow;
+  unsigned int sat8, sat16, gt1;
+};
+struct RowState {
+  float mu[4];
+  float om[4];
+};
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+// Byte address of (row, 16-byte chunk) inside a [rows][64] bf16 tile with the 128-byte swizzle.
+__device__ __forceinline__ uint32_t sw128(int row, int chunk) { return row * 128 + ((chunk ^ (row & 7)) << 4); }
+
+// Everything between the low-precision logits and the P V product of Alg. 1 for one
+// (group, key tile): threats and order, stage 1 (eq. (7)), exponentials, lambda / omega,
+// stage 2 (eq. (8)), stage-2 recomputation.  Writes the group's 32 rows of the P tile
+// (bf16 hi, and bf16 lo for 16-bit sub-blocks), returns the flag byte.
+template <int D, bool FULL, bool DUMP>
+__device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileGeom& g, float (&acc)[4][16],
+                                              const float* kf, const __nv_bfloat16* qrow, const uint32_t* lut,
+                                              unsigned char* phi, unsigned char* plo, uint32_t tscratch,
+                                              uint32_t& lo_dirty, RowState& st, float (&lam)[4],
+                                              WarpCounters& wc, unsigned long long (&cks)[2], int dump_row0,
+                                              int row0) {
+  const int lane = threadIdx.x & 31;
+  const int qa = lane >> 2, th_own = lane & 3;
+  const double scale_d = (double)P.scale;
+  const bool force16 = P.flags & LAMP_FORCE_16BIT;
+  const bool force8 = P.flags & LAMP_FORCE_8BIT;
+  const bool skip1 = (P.flags & (LAMP_FORCE_8BIT | LAMP_NO_STAGE1)) != 0;
+
+  // ---- per sub-block, per query maxima; which sub-blocks are active ----------------------
+  float cm[4];
+#pragma unroll
+  for (int a = 0; a < 4; ++a) {
+    float m = -INFINITY;
+#pragma unroll
+    for (int b = 0; b < 16; ++b)
+      if (vis<FULL>(g, 16 * th_own + b, 4 * qa + a)) m = fmaxf(m, acc[a][b]);
+    cm[a] = m;
+  }
+  uint32_t actmask = 0;
+#pragma unroll
+  for (int th = 0; th < 4; ++th) {
+    bool act = true;
+    if (!FULL) {
+      const int s0 = g.i0 + 16 * th;
+      act = (!g.causal || s0 <= g.j0 + 31) && (g.window == 0 || g.j0 - (s0 + 15) < g.window);
+    }
+    actmask |= (uint32_t)act << th;
+  }
+  const int nact = __popc(actmask);
+
+  // ---- threats T_theta against the maxima at tile start, visiting order ------------------
+  float tl = -INFINITY;
+#pragma unroll
+  for (int a = 0; a < 4; ++a)
+    if (cm[a] > -INFINITY) tl = fmaxf(tl, __fsub_rn(cm[a], st.mu[a]));
+  tl = fmaxf(tl, __shfl_xor_sync(kFull, tl, 4));
+  tl = fmaxf(tl, __shfl_xor_sync(kFull, tl, 8));
+  tl = fmaxf(tl, __shfl_xor_sync(kFull, tl, 16));
+  float T[4];
+#pragma unroll
+  for (int th = 0; th < 4; ++th) T[th] = __shfl_sync(kFull, tl, th);
+  uint32_t order = 0;   // 2 bits per rank: the sub-block visited at that rank
+#pragma unroll
+  for (int th = 0; th < 4; ++th) {
+    int rank = 0;
+#pragma unroll
+    for (int o = 0; o < 4; ++o)
+      if (o != th && ((actmask >> o) & 1u) && (T[o] > T[th] || (T[o] == T[th] && o < th))) ++rank;
+    if ((actmask >> th) & 1u) order |= (uint32_t)th << (2 * rank);
+  }
+
+  // ---- stage 1: eq. (7), sub-blocks in threat order ----------------------------------------
+  float muh[4];
+#pragma unroll
+  for (int a = 0; a < 4; ++a) muh[a] = st.mu[a];
+  uint32_t Theta = 0;
+  for (int r = 0; r < nact; ++r) {
+    const int th = (order >> (2 * r)) & 3;
+    bool fail;
+    if (force16) fail = true;
+    else if (skip1) fail = false;
+    else {
+      bool f = false;
+      if (th_own == th) {
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+          if (cm[a] > -INFINITY) {
+            const float rhs = __fadd_rn(cm[a], __fmul_rn(fabsf(muh[a]), P.delta));
+            if (isinf(muh[a]) || !(muh[a] > rhs)) f = true;
+          }
+      }
+      fail = __any_sync(kFull, f);
+    }
+    if (!fail) continue;
+    Theta |= 1u << th;
+    float y[4][4];
+    dot16<D>(kf, qrow, P.qs[2], th, th_own, scale_d, y);
+    uint32_t yr[16];
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+      float m = -INFINITY;
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        yr[4 * a + b] = __float_as_uint(y[a][b]);
+        if (vis<FULL>(g, 16 * th + 4 * th_own + b, 4 * qa + a)) {
+          m = fmaxf(m, y[a][b]);
+          wc.sat16 += fabsf(y[a][b]) == 448.0f;
+        }
+      }
+      m = fmaxf(m, __shfl_xor_sync(kFull, m, 1));
+      m = fmaxf(m, __shfl_xor_sync(kFull, m, 2));
+      muh[a] = fmaxf(muh[a], m);
+    }
+    ptx::tmem_st16(tscratch + 16 * th, yr);   // parked in this thread's own TMEM lane
+  }
+  if (Theta) ptx::tmem_wait_st();
+  if (skip1 && !force16) {
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+      float m = cm[a];
+      m = fmaxf(m, __shfl_xor_sync(kFull, m, 1));
+      m = fmaxf(m, __shfl_xor_sync(kFull, m, 2));
+      muh[a] = fmaxf(muh[a], m);
+    }
+  }
+
+  // ---- exponentials: 8-bit through the table, 16-bit correctly rounded -----------------------
+  const bool own_act = (actmask >> th_own) & 1u;
+  const bool own8 = own_act && !((Theta >> th_own) & 1u);
+  double rs8[4] = {0.0, 0.0, 0.0, 0.0};
+  if (own_act) {
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+      const float m8 = trunc_e4m3(muh[a]);
+#pragma unroll
+      for (int b = 0; b < 16; ++b) {
+        const bool ok = vis<FULL>(g, 16 * th_own + b, 4 * qa + a);
+        float e = 0.0f;
+        if (ok) {
+          const float y8 = acc[a][b];
+          uint32_t eb = 0xffu;
+          wc.sat8 += fabsf(y8) == 448.0f;
+          if (own8) {
+            const uint32_t w = lut[shift_index(__fsub_rn(m8, y8))];
+            e = __uint_as_float(w & 0xffffff00u);
+            eb = w & 0xffu;
+          }
+          if (DUMP) {
+            const uint32_t yb = enc_e4m3(y8);
+            const uint64_t idx = (uint64_t)((16 * th_own + b) * kBQ + 4 * qa + a) << 8;
+            cks[0] += mix64(idx | yb);
+            cks[1] += mix64(idx | eb);
+            if (dump_row0 >= 0) {
+              const size_t off = (size_t)(dump_row0 + 4 * qa + a) * P.seqlen + g.i0 + 16 * th_own + b;
+              if (P.dbg_y8) P.dbg_y8[off] = (uint8_t)yb;
+              if (P.dbg_e8) P.dbg_e8[off] = (uint8_t)eb;
+            }
+          }
+        }
+        acc[a][b] = e;
+        rs8[a] += (double)e;
+      }
+    }
+  } else {
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+      for (int b = 0; b < 16; ++b) acc[a][b] = 0.0f;
+  }
+
+  // 16-bit exponentials of sub-block th for this lane's (quad x 4 keys); written straight
+  // into the P tile as bf16 hi + lo (12 significant bits = 8 + a remainder of at most 5).
+  double rs16[4] = {0.0, 0.0, 0.0, 0.0};
+  auto exp_block = [&](int th, const float (&y)[4][4]) {
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+      float e[4], h[4], l[4];
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        e[b] = 0.0f;
+        if (vis<FULL>(g, 16 * th + 4 * th_own + b, 4 * qa + a)) {
+          e[b] = exp16(rne_sig12(__fsub_rn(y[a][b], muh[a])));
+          wc.gt1 += e[b] > 1.0f;
+        }
+        rs16[a] += (double)e[b];
+        h[b] = __bfloat162float(__float2bfloat16_rn(e[b]));
+        l[b] = e[b] - h[b];
+      }
+      const int row = row0 + 4 * qa + a;
+      const uint32_t off = sw128(row, 2 * th + (th_own >> 1)) + (th_own & 1) * 8;
+      *reinterpret_cast<uint2*>(phi + off) = make_uint2(pack_bf16(h[0], h[1]), pack_bf16(h[2], h[3]));
+      *reinterpret_cast<uint2*>(plo + off) = make_uint2(pack_bf16(l[0], l[1]), pack_bf16(l[2], l[3]));
+    }
+  };
+  for (int th = 0; th < 4; ++th) {
+    if (!((Theta >> th) & 1u)) continue;
+    uint32_t yr[16];
+    ptx::tmem_ld16(tscratch + 16 * th, yr);
+    ptx::tmem_wait_ld();
+    float y[4][4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+      for (int b = 0; b < 4; ++b) y[a][b] = __uint_as_float(yr[4 * a + b]);
+    exp_block(th, y);
+  }
+
+  // ---- lambda_hat (one high-precision exponential per row), omega_hat ------------------------
+  double lw[4];
+  float omh[4];
+  bool big = false;
+#pragma unroll
+  for (int a = 0; a < 4; ++a) {
+    lam[a] = isinf(st.mu[a]) ? 0.0f : (float)exp((double)__fsub_rn(st.mu[a], muh[a]));
+    lw[a] = __dmul_rn((double)lam[a], (double)st.om[a]);
+    double R = (own8 ? rs8[a] : 0.0) + rs16[a];
+    R += shfl_xor_d(R, 1);
+    R += shfl_xor_d(R, 2);
+    big |= !(R < 4096.0);
+    omh[a] = (float)__dadd_rn(lw[a], R);
+  }
+
+  // ---- stage 2: block-LAMP problem, eq. (8) -----------------------------------------------------
+  const uint32_t freem = actmask & ~Theta;
+  uint32_t Rset = 0;
+  if (!force8 && !force16 && freem) {
+    double xi[4] = {0.0, 0.0, 0.0, 0.0};
+    if (own8) {
+#pragma unroll
+      for (int a = 0; a < 4; ++a) {
+        const double oh = (double)omh[a];
+#pragma unroll
+        for (int b = 0; b < 16; ++b) {
+          const double e = (double)acc[a][b];   // invisible pairs hold 0 and add exactly +0
+          xi[a] = __dadd_rn(xi[a], __dmul_rn(__dsub_rn(oh, e), e));
+        }
+      }
+    }
+    uint32_t feas = 0xffffu;
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+      double x[4];
+#pragma unroll
+      for (int th = 0; th < 4; ++th) x[th] = shfl_d(xi[a], (lane & ~3) | th);
+      const double oh = (double)omh[a];
+      const double rhs = __dmul_rn(__dmul_rn((double)P.tau, oh), oh);
+#pragma unroll
+      for (uint32_t r = 0; r < 16; ++r) {
+        const uint32_t keep = freem & ~r;
+        double kept = 0.0;
+#pragma unroll
+        for (int th = 0; th < 4; ++th)
+          if ((keep >> th) & 1u) kept = __dadd_rn(kept, x[th]);
+        if (!(kept <= rhs)) feas &= ~(1u << r);
+      }
+    }
+    feas = __reduce_and_sync(kFull, feas);
+    int best = 5;   // smallest recompute set, then smallest bitmask, among subsets of the free ones
+#pragma unroll
+    for (uint32_t r = 0; r < 16; ++r) {
+      const int sz = __popc(r);
+      if ((r & ~freem) == 0 && ((feas >> r) & 1u) && sz < best) { best = sz; Rset = r; }
+    }
+  }
+
+  // ---- stage-2 recomputation with the maxima unchanged -------------------------------------------
+  for (int th = 0; th < 4; ++th) {
+    if (!((Rset >> th) & 1u)) continue;
+    float y[4][4];
+    dot16<D>(kf, qrow, P.qs[2], th, th_own, scale_d, y);
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+      for (int b = 0; b < 4; ++b)
+        if (vis<FULL>(g, 16 * th + 4 * th_own + b, 4 * qa + a)) wc.sat16 += fabsf(y[a][b]) == 448.0f;
+    exp_block(th, y);
+  }
+
+  // ---- state update ------------------------------------------------------------------------------
+  const bool keep8 = own8 && !((Rset >> th_own) & 1u);
+#pragma unroll
+  for (int a = 0; a < 4; ++a) {
+    double R = (keep8 ? rs8[a] : 0.0) + rs16[a];
+    R += shfl_xor_d(R, 1);
+    R += shfl_xor_d(R, 2);
+    big |= !(R < 4096.0);
+    st.mu[a] = muh[a];
+    st.om[a] = (float)__dadd_rn(lw[a], R);
+  }
+  // 8-bit exponentials that stay (4 significant bits: exact in bf16) and zeros of inactive
+  // sub-blocks; the lo tile is zero wherever this group has no 16-bit sub-block.
+  const uint32_t hi16 = Theta | Rset;
+  if (keep8 || !own_act) {
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+      const int row = row0 + 4 * qa + a;
+      uint32_t w[8];
+#pragma unroll
+      for (int b = 0; b < 8; ++b) w[b] = pack_bf16(acc[a][2 * b], acc[a][2 * b + 1]);
+      *reinterpret_cast<uint4*>(phi + sw128(row, 2 * th_own)) = make_uint4(w[0], w[1], w[2], w[3]);
+      *reinterpret_cast<uint4*>(phi + sw128(row, 2 * th_own + 1)) = make_uint4(w[4], w[5], w[6], w[7]);
+    }
+  }
+  if (((lo_dirty & ~hi16) >> th_own) & 1u) {
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+      const int row = row0 + 4 * qa + a;
+      *reinterpret_cast<uint4*>(plo + sw128(row, 2 * th_own)) = make_uint4(0, 0, 0, 0);
+      *reinterpret_cast<uint4*>(plo + sw128(row, 2 * th_own + 1)) = make_uint4(0, 0, 0, 0);
+    }
+  }
+  lo_dirty = hi16;
+
+  if (__any_sync(kFull, big)) wc.bigrow++;
+  wc.active += nact;
+  wc.s1 += __popc(Theta);
+  wc.s2 += __popc(Rset);
+  wc.hist[__popc(hi16)]++;
+  return Theta | (Rset << 4);
+}
+
+template <int D, bool DUMP>
+__global__ void __launch_bounds__(kThreads, 1)
+lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ CUtensorMap kmap,
+               const __grid_constant__ CUtensorMap vmap, const uint32_t* __restrict__ lut_g,
+               DeviceStats* __restrict__ gstats) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
+  using L = Smem<D>;
+  float* qsT = reinterpret_cast<float*>(smem + L::kQs);
+  float* kf_all = reinterpret_cast<float*>(smem + L::kKf);
+  unsigned char* kbf = smem + L::kKbf;
+  unsigned char* vs = smem + L::kV;
+  unsigned char* phi = smem + L::kPhi;
+  unsigned char* plo = smem + L::kPlo;
+  uint32_t* lut = reinterpret_cast<uint32_t*>(smem + L::kLut);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBar);
+  uint32_t* tslot = reinterpret_cast<uint32_t*>(smem + L::kMisc);
+  uint32_t* lomask = tslot + 1;   // [2]
+  int* status = &gstats->status;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int ntq = P.seqlen / kBM;
+  const int qt = ntq - 1 - (int)blockIdx.x;   // long (late) query tiles first
+  const int h = blockIdx.y, b = blockIdx.z;
+  const int hk = h / (P.heads_q / P.heads_kv);
+  const int m0 = qt * kBM;
+
+  int t_begin = 0, t_end = P.seqlen / kTK;
+  if (P.causal) t_end = min(t_end, (m0 + kBM - 1) / kTK + 1);
+  if (P.window > 0) t_begin = max(0, m0 - P.window + 1) / kTK;
+  const int T = t_end - t_begin;
+
+  // ---- set-up ---------------------------------------------------------------------------------
+  if (tid == 0) {
+    ptx::mbar_init(&bars[kKbfFull], 1);
+    ptx::mbar_init(&bars[kKbfEmpty], kConvWarps);
+    ptx::mbar_init(&bars[kKfFull0], kConvWarps);
+    ptx::mbar_init(&bars[kKfFull1], kConvWarps);
+    ptx::mbar_init(&bars[kKfEmpty0], 4);
+    ptx::mbar_init(&bars[kKfEmpty1], 4);
+    ptx::mbar_init(&bars[kVFull], 1);
+    ptx::mbar_init(&bars[kPReady], 4);
+    ptx::mbar_init(&bars[kPvDone], 1);
+    ptx::fence_barrier_init();
+    lomask[0] = lomask[1] = 0;
+  }
+  if (warp == kCtrlWarp) {
+    ptx::tmem_alloc(tslot, 256);
+    ptx::tmem_relinquish();
+    if (lane == 0) { ptx::prefetch_tensormap(&kmap); ptx::prefetch_tensormap(&vmap); }
+  }
+  for (int i = tid; i < 256; i += kThreads) lut[i] = lut_g[i];
+  {
+    const __nv_bfloat16* qg = P.q + b * P.qs[0] + h * P.qs[1] + (int64_t)m0 * P.qs[2];
+    for (int c = tid; c < kBM * D / 8; c += kThreads) {
+      const int row = c % kBM, k0 = (c / kBM) * 8;   // consecutive threads -> consecutive rows
+      const uint4 raw = *reinterpret_cast<const uint4*>(qg + (int64_t)row * P.qs[2] + k0);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const uint32_t w = (&raw.x)[e >> 1];
+        const float f = __uint_as_float((e & 1) ? (w & 0xffff0000u) : (w << 16));
+        qsT[(k0 + e) * kBM + row] = __fmul_rn(f, P.scale);
+      }
+    }
+    for (int c = tid; c < kBM * kTK * 2 / 16; c += kThreads) {
+      reinterpret_cast<uint4*>(phi)[c] = make_uint4(0, 0, 0, 0);
+      reinterpret_cast<uint4*>(plo)[c] = make_uint4(0, 0, 0, 0);
+    }
+  }
+  ptx::fence_proxy_async();
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tbase = *tslot;
+
+  if (warp == kCtrlWarp) {
+    // =========================== control: TMA loads and MMA issue ================================
+    // (all 32 lanes walk the loop so that the warp stays converged; lane 0 issues)
+    constexpr uint32_t kTileBytes = kTK * D * 2;
+    constexpr uint32_t idesc = ptx::idesc_bf16(kBM, D, 1);
+    bool ok = true;
+    if (lane == 0) {
+      ptx::mbar_arrive_expect_tx(&bars[kKbfFull], kTileBytes);
+      ptx::mbar_arrive_expect_tx(&bars[kVFull], kTileBytes);
+#pragma unroll
+      for (int x = 0; x < D / 64; ++x) {
+        ptx::tma_load_4d(kbf + x * 8192, &kmap, &bars[kKbfFull], 64 * x, t_begin * kTK, hk, b);
+        ptx::tma_load_4d(vs + x * 8192, &vmap, &bars[kVFull], 64 * x, t_begin * kTK, hk, b);
+      }
+    }
+    __syncwarp();
+    for (int n = 0; n < T && ok; ++n) {
+      if (n + 1 < T) {
+        ok = ptx::mbar_wait(&bars[kKbfEmpty], n & 1, status, kTimeoutCode);
+        if (lane == 0 && ok) {
+          ptx::mbar_arrive_expect_tx(&bars[kKbfFull], kTileBytes);
+#pragma unroll
+          for (int x = 0; x < D / 64; ++x)
+            ptx::tma_load_4d(kbf + x * 8192, &kmap, &bars[kKbfFull], 64 * x, (t_begin + n + 1) * kTK, hk, b);
+        }
+      }
+      ok = ok && ptx::mbar_wait(&bars[kPReady], n & 1, status, kTimeoutCode);
+      ok = ok && ptx::mbar_wait(&bars[kVFull], n & 1, status, kTimeoutCode);
+      ok = __all_sync(kFull, ok);
+      ptx::tc_fence_after();
+      if (lane == 0 && ok) {
+        const uint32_t lom = lomask[n & 1];
+        lomask[n & 1] = 0;
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks) {
+          const uint64_t bd = ptx::smem_desc_sw128(ptx::smem_u32(vs) + ks * 2048, 8192, 1024);
+          ptx::umma_bf16(tbase, ptx::smem_desc_sw128(ptx::smem_u32(phi) + ks * 32, 16, 1024), bd, idesc,
+                         (n > 0 || ks > 0) ? 1u : 0u);
+          if ((lom >> ks) & 1u)
+            ptx::umma_bf16(tbase, ptx::smem_desc_sw128(ptx::smem_u32(plo) + ks * 32, 16, 1024), bd, idesc, 1u);
+        }
+        ptx::umma_commit(&bars[kPvDone]);
+      }
+      __syncwarp();
+      if (n + 1 < T && ok) {
+        ok = ptx::mbar_wait(&bars[kPvDone], n & 1, status, kTimeoutCode);
+        if (lane == 0 && ok) {
+          ptx::mbar_arrive_expect_tx(&bars[kVFull], kTileBytes);
+#pragma unroll
+          for (int x = 0; x < D / 64; ++x)
+            ptx::tma_load_4d(vs + x * 8192, &vmap, &bars[kVFull], 64 * x, (t_begin + n + 1) * kTK, hk, b);
+        }
+      }
+      ok = __all_sync(kFull, ok);
+    }
+  } else if (warp >= 4) {
+    // =========================== converters: bf16 K tile -> fp32, key-contiguous ===================
+    const int key = tid - 128;         // 0..63: one key of the tile per thread
+    bool ok = true;
+    for (int n = 0; n < T && ok; ++n) {
+      float* kf = kf_all + (n & 1) * D * kKfStride;
+      ok = ptx::mbar_wait(&bars[kKbfFull], n & 1, status, kTimeoutCode);
+      if (n >= 2) ok = ok && ptx::mbar_wait(&bars[kKfEmpty0 + (n & 1)], ((n >> 1) - 1) & 1, status, kTimeoutCode);
+      const int pos = kf_pos(key);
+#pragma unroll 4
+      for (int c = 0; c < D / 8; ++c) {   // 16-byte chunk c: channels 8c..8c+7 of this key
+        const int box = c >> 3, cc = c & 7;
+        const uint4 raw = *reinterpret_cast<const uint4*>(kbf + box * 8192 + sw128(key, cc));
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const uint32_t w = (&raw.x)[e >> 1];
+          kf[(8 * c + e) * kKfStride + pos] = __uint_as_float((e & 1) ? (w & 0xffff0000u) : (w << 16));
+        }
+      }
+      __syncwarp();
+      if (lane == 0) {
+        ptx::mbar_arrive(&bars[kKfFull0 + (n & 1)]);
+        ptx::mbar_arrive(&bars[kKbfEmpty]);
+      }
+    }
+  } else {
+    // =========================== compute: one group of 32 query rows per warp =====================
+    const int qa = lane >> 2;
+    const int j0 = m0 + warp * kBQ;
+    const int ntk = P.seqlen / kTK;
+    const bool dump_rows = DUMP && b == P.dbg_batch && h == P.dbg_head;
+    const __nv_bfloat16* qrow = P.q + b * P.qs[0] + h * P.qs[1] + (int64_t)(j0 + 4 * qa) * P.qs[2];
+    const uint32_t tlane = tbase + ((uint32_t)(warp * 32) << 16);
+    RowState st;
+#pragma unroll
+    for (int a = 0; a < 4; ++a) { st.mu[a] = -INFINITY; st.om[a] = 0.0f; }
+    WarpCounters wc;
+    memset(&wc, 0, sizeof(wc));
+    uint32_t lo_dirty = 0;
+    bool ok = true;
+
+    for (int n = 0; n < T && ok; ++n) {
+      const int t = t_begin + n, i0 = t * kTK;
+      const float* kf = kf_all + (n & 1) * D * kKfStride;
+      TileGeom g;
+      g.i0 = i0; g.j0 = j0; g.causal = P.causal; g.window = P.window;
+      const bool any = (!P.causal || i0 <= j0 + 31) && (P.window == 0 || j0 - (i0 + 63) < P.window);
+      const bool full = (!P.causal || i0 + 63 <= j0) && (P.window == 0 || (j0 + 31) - i0 < P.window);
+      float lam[4] = {1.0f, 1.0f, 1.0f, 1.0f};
+      uint32_t flag = 0;
+      unsigned long long cks[2] = {0ull, 0ull};
+
+      ok = ptx::mbar_wait(&bars[kKfFull0 + (n & 1)], (n >> 1) & 1, status, kTimeoutCode);
+      float acc[4][16];
+      if (any) chain8<D>(qsT + warp * kBQ + 4 * qa, kf + kf_pos(16 * (lane & 3)), acc);
+      // the previous P V product must be complete before O is rescaled or P is overwritten
+      if (n > 0) ok = ok && ptx::mbar_wait(&bars[kPvDone], (n - 1) & 1, status, kTimeoutCode);
+      ptx::tc_fence_after();
+      if (any) {
+        const int dump0 = dump_rows ? j0 : -1;
+        if (full)
+          flag = lamp_post<D, true, DUMP>(P, g, acc, kf, qrow, lut, phi, plo, tlane + D, lo_dirty, st, lam, wc,
+                                          cks, dump0, warp * kBQ);
+        else
+          flag = lamp_post<D, false, DUMP>(P, g, acc, kf, qrow, lut, phi, plo, tlane + D, lo_dirty, st, lam, wc,
+                                           cks, dump0, warp * kBQ);
+      } else {
+        // no visible pair for this group: its rows of the P tile are zero
+        for (int c = lane; c < kBQ * 8; c += 32) {
+          *reinterpret_cast<uint4*>(phi + sw128(warp * kBQ + (c >> 3), c & 7)) = make_uint4(0, 0, 0, 0);
+          if (lo_dirty) *reinterpret_cast<uint4*>(plo + sw128(warp * kBQ + (c >> 3), c & 7)) = make_uint4(0, 0, 0, 0);
+        }
+        lo_dirty = 0;
+      }
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&bars[kKfEmpty0 + (n & 1)]);
+
+      // O <- diag(lambda_hat) O, only when some row of the group changes its maximum
+      bool resc = false;
+#pragma unroll
+      for (int a = 0; a < 4; ++a) resc |= lam[a] != 1.0f;
+      if (n > 0 && __any_sync(kFull, resc)) {
+        float lrow = 1.0f;   // lambda of the row this lane owns in TMEM (row = lane)
+#pragma unroll
+        for (int a = 0; a < 4; ++a) {
+          const float v = __shfl_sync(kFull, lam[a], (lane >> 2) << 2);
+          if ((lane & 3) == a) lrow = v;
+        }
+#pragma unroll 1
+        for (int c0 = 0; c0 < D; c0 += 16) {
+          uint32_t r[16];
+          ptx::tmem_ld16(tlane + c0, r);
+          ptx::tmem_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * lrow);
+          ptx::tmem_st16(tlane + c0, r);
+        }
+        ptx::tmem_wait_st();
+      }
+      const uint32_t lo_now = (flag | (flag >> 4)) & 15u;
+      if (lane == 0 && lo_now) atomicOr(&lomask[n & 1], lo_now);
+      ptx::fence_proxy_async();
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&bars[kPReady]);
+
+      const int64_t gt = (((int64_t)b * P.heads_q + h) * (P.seqlen / kBQ) + (j0 / kBQ)) * ntk + t;
+      if (lane == 0 && P.flag_mask) P.flag_mask[gt] = (uint8_t)flag;
+      if (DUMP && P.dbg_checksums) {
+#pragma unroll
+        for (int s = 16; s > 0; s >>= 1) {
+          cks[0] += __shfl_xor_sync(kFull, cks[0], s);
+          cks[1] += __shfl_xor_sync(kFull, cks[1], s);
+        }
+        if (lane == 0) { P.dbg_checksums[2 * gt] = cks[0]; P.dbg_checksums[2 * gt + 1] = cks[1]; }
+      }
+    }
+
+    // ---- epilogue: O / omega, lse = mu + ln(omega) ------------------------------------------------
+    if (T > 0) ok = ok && ptx::mbar_wait(&bars[kPvDone], (T - 1) & 1, status, kTimeoutCode);
+    ptx::tc_fence_after();
+    float om_row = 1.0f, mu_row = 0.0f;
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+      const float o = __shfl_sync(kFull, st.om[a], (lane >> 2) << 2);
+      const float m = __shfl_sync(kFull, st.mu[a], (lane >> 2) << 2);
+      if ((lane & 3) == a) { om_row = o; mu_row = m; }
+    }
+    // lane l holds row j0 + l of O: rows 4*(l>>2) + (l&3)
+    const int64_t orow = b * P.os[0] + h * P.os[1] + (int64_t)(j0 + lane) * P.os[2];
+    if (P.lse) P.lse[((int64_t)b * P.heads_q + h) * P.seqlen + j0 + lane] = (float)((double)mu_row + log((double)om_row));
+#pragma unroll 1
+    for (int c0 = 0; c0 < D; c0 += 16) {
+      uint32_t r[16];
+      ptx::tmem_ld16(tlane + c0, r);
+      ptx::tmem_wait_ld();
+      if (P.flags & LAMP_OUT_FP32) {
+        float* dst = reinterpret_cast<float*>(P.out) + orow + c0;
+#pragma unroll
+        for (int i = 0; i < 16; i += 4)
+          *reinterpret_cast<float4*>(dst + i) =
+              make_float4(__uint_as_float(r[i]) / om_row, __uint_as_float(r[i + 1]) / om_row,
+                          __uint_as_float(r[i + 2]) / om_row, __uint_as_float(r[i + 3]) / om_row);
+      } else {
+        __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(P.out) + orow + c0;
+        uint32_t w[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          w[i] = pack_bf16(__uint_as_float(r[2 * i]) / om_row, __uint_as_float(r[2 * i + 1]) / om_row);
+        *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+        *reinterpret_cast<uint4*>(dst + 8) = make_uint4(w[4], w[5], w[6], w[7]);
+      }
+    }
+
+    // ---- counters -----------------------------------------------------------------------------------
+    const unsigned sat8 = __reduce_add_sync(kFull, wc.sat8);
+    const unsigned sat16 = __reduce_add_sync(kFull, wc.sat16);
+    const unsigned gt1 = __reduce_add_sync(kFull, wc.gt1);
+    if (lane == 0) {
+      atomicAdd(&gstats->v[0], wc.active);
+      atomicAdd(&gstats->v[1], wc.s1);
+      atomicAdd(&gstats->v[2], wc.s2);
+#pragma unroll
+      for (int i = 0; i < 5; ++i) atomicAdd(&gstats->v[3 + i], wc.hist[i]);
+      atomicAdd(&gstats->v[8], (unsigned long long)sat8);
+      atomicAdd(&gstats->v[9], (unsigned long long)sat16);
+      atomicAdd(&gstats->v[10], (unsigned long long)gt1);
+      atomicAdd(&gstats->v[11], wc.bigrow);
+    }
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == kCtrlWarp) ptx::tmem_dealloc(tbase, 256);
+}
+
+}  // namespace lamp
