@@ -157,6 +157,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--mode", default="lamp", choices=["lamp", "force8", "force16"],
+                    help="internal comparison modes: pure 8-bit / every sub-block 16-bit")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -195,6 +197,7 @@ def main():
     p.batch, p.heads_q, p.heads_kv, p.seqlen, p.head_dim = B, Hq, k.shape[1], N, D
     lamp.lamp_attn_contiguous_strides(p)
     p.causal, p.scale = 1, scale
+    p.flags = {"lamp": 0, "force8": lamp.LAMP_FORCE_8BIT, "force16": lamp.LAMP_FORCE_16BIT}[args.mode]
     fl = flops_of(cfg)
 
     def step():
@@ -287,7 +290,7 @@ def main():
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "e4m3-emulated/f32", "data": "synthetic", "config": workload_config(cfg),
-            "clocks": clk.summary(),
+            "mode": args.mode, "clocks": clk.summary(),
             "e2e": {"value": world * fl / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
             "gpu_launches": args.steps,

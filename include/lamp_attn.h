@@ -80,12 +80,17 @@ typedef struct lamp_attn_stats {
   uint64_t stage2_flagged;           /* recomputed by the solution of eq. (8)                  */
   uint64_t hist_flagged_per_tile[5]; /* (group, key tile) pairs with 0..4 recomputed sub-blocks:
                                         the "16-bit sub-blocks per tile" columns of Tables 1-6 */
-  uint64_t sat_e4m3;                 /* visible pairs whose 8-bit logit ended at +-448         */
+  uint64_t sat_e4m3;                 /* (sub-block, query) pairs whose largest 8-bit logit is 448 */
   uint64_t sat_e4m11;                /* recomputed pairs whose 16-bit logit ended at +-448     */
   uint64_t exp16_gt1;                /* 16-bit exponentials above 1 (stage-2 logit > maximum)  */
   uint64_t big_rowsum;               /* (group, tile) pairs with a row sum of 2^12 or more     */
   int32_t device_status;             /* 0, or LAMP_ERR_DEVICE_TIMEOUT                          */
   int32_t reserved;
+  uint64_t phase_cycles[8];          /* profiling aid, all zero unless the library was built with
+                                        -DLAMP_PHASE_TIMERS: SM cycles summed over the compute warps
+                                        in [0] wait for K, [1] 8-bit chain, [2] wait for P V,
+                                        [3] decision path total, [4] 16-bit logits, [5] 16-bit
+                                        exponentials, [6] stage 2, [7] rescale and hand-off       */
 } lamp_attn_stats;
 
 /* Fill *p with zeros and the paper's defaults (tau = 0.5, delta = 2^-8, causal = 1,

@@ -295,6 +295,7 @@ static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
         for (int i = th * BK; i < (th + 1) * BK; ++i)
           if (val[i][j] && Y8[i][j] > m) m = Y8[i][j];
         cm8[th][j] = m;
+        if (m == 448.0f) st->sat_e4m3++;
       }
 
     /* threats T_theta against the maxima at tile start, then the visiting order */
@@ -401,7 +402,6 @@ static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
       for (int j = 0; j < BQ; ++j) {
         if (!val[i][j]) continue;
         uint8_t yb = lamp_oracle_enc_e4m3(Y8[i][j]);
-        if (fabsf(Y8[i][j]) == 448.0f) st->sat_e4m3++;
         if (y8d) y8d[(size_t)j * N + i0 + i] = yb;
         if (e8d) e8d[(size_t)j * N + i0 + i] = E8[i][j];
         if (checks) {

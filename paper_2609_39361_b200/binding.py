@@ -32,12 +32,14 @@ class LampAttnStats(C.Structure):
     _fields_ = [("subblocks_active", C.c_uint64), ("stage1_flagged", C.c_uint64),
                 ("stage2_flagged", C.c_uint64), ("hist_flagged_per_tile", C.c_uint64 * 5),
                 ("sat_e4m3", C.c_uint64), ("sat_e4m11", C.c_uint64), ("exp16_gt1", C.c_uint64),
-                ("big_rowsum", C.c_uint64), ("device_status", C.c_int32), ("reserved", C.c_int32)]
+                ("big_rowsum", C.c_uint64), ("device_status", C.c_int32), ("reserved", C.c_int32),
+                ("phase_cycles", C.c_uint64 * 8)]
 
     def as_dict(self):
         d = {k: int(getattr(self, k)) for k, _ in self._fields_
-             if k not in ("hist_flagged_per_tile", "reserved")}
+             if k not in ("hist_flagged_per_tile", "reserved", "phase_cycles")}
         d["hist_flagged_per_tile"] = [int(x) for x in self.hist_flagged_per_tile]
+        d["phase_cycles"] = [int(x) for x in self.phase_cycles]
         return d
 
 

@@ -22,7 +22,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     deps = [d for d in DEPS if os.path.exists(d)]
     if not force and os.path.exists(LIB) and all(os.path.getmtime(LIB) >= os.path.getmtime(d) for d in deps):
         return LIB
-    cmd = ["nvcc"] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + [SRC, "-o", LIB]
+    extra = ["-DLAMP_PHASE_TIMERS=" + os.environ["LAMP_PHASE_TIMERS"]] if os.environ.get("LAMP_PHASE_TIMERS") else []
+    cmd = ["nvcc"] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + [SRC, "-o", LIB]
     subprocess.check_call(cmd)
     return LIB
 

@@ -10,7 +10,7 @@
 namespace lamp {
 
 __device__ DeviceStats g_stats;
-__device__ uint32_t g_lut8[256];   // fp32 bits of the 8-bit exponential | its byte
+__device__ uint2 g_lut8[128];   // .x = fp32 bits of the 8-bit exponential, .y = the same if below 2^-15, else 0
 
 typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                       const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
@@ -68,12 +68,21 @@ static int ensure_device(int* dev_out) {
   e = cudaGetDeviceProperties(&prop, dev);
   if (e != cudaSuccess) return cuda_fail(e);
   if (prop.major != 10) return LAMP_ERR_UNSUPPORTED_DEVICE;
-  // table index = shift byte (ue5m3, bias 15): value 2^(E-15)(1 + M/8), E = 0: 2^-14 M/8
-  uint32_t lut[256];
-  for (int p = 0; p < 256; ++p) {
-    const int E = p >> 3, M = p & 7;
-    const double s = E ? ldexp(1.0 + M / 8.0, E - 15) : ldexp(M / 8.0, -14);
-    lut[p] = exp8_entry(s);
+  // The 256-entry table of Sec. 3.3 maps the shift (4 significant bits) to the correctly
+  // rounded 8-bit exponential.  The kernel indexes it by the e4m3 code c of HALF the shift,
+  // which the conversion unit produces: for shift/2 >= 2^-6 that code holds exactly the
+  // 4-significant-bit rounding of the shift; below it (shift < 2^-5) every entry is 1.0
+  // in both indexings, so the two tables agree on every shift that can occur.
+  uint2 lut[128];
+  for (int c = 0; c < 128; ++c) {
+    const int E = c >> 3, M = c & 7;
+    const double half = E ? ldexp(1.0 + M / 8.0, E - 7) : ldexp(M / 8.0, -6);
+    const uint32_t w = exp8_entry(2.0 * half);
+    const uint32_t vbits = w & 0xffffff00u;
+    float vf;
+    memcpy(&vf, &vbits, 4);
+    lut[c].x = vbits;
+    lut[c].y = vf < ldexp(1.0f, -15) ? vbits : 0u;
   }
   e = cudaMemcpyToSymbol(g_lut8, lut, sizeof(lut));
   if (e != cudaSuccess) return cuda_fail(e);
@@ -221,10 +230,10 @@ int lamp_attn_fwd(const void* q, const void* k, const void* v, void* out, float*
   const bool dump = p->dbg_y8 || p->dbg_e8 || p->dbg_checksums;
   dim3 grid(p->seqlen / kBM, p->heads_q, p->batch), block(kThreads);
   if (dump)
-    lamp_fwd_sm100<128, true><<<grid, block, kSmemLaunch128, stream>>>(P, kmap, vmap, (const uint32_t*)lut_ptr,
+    lamp_fwd_sm100<128, true><<<grid, block, kSmemLaunch128, stream>>>(P, kmap, vmap, (const uint2*)lut_ptr,
                                                                        (DeviceStats*)stats_ptr);
   else
-    lamp_fwd_sm100<128, false><<<grid, block, kSmemLaunch128, stream>>>(P, kmap, vmap, (const uint32_t*)lut_ptr,
+    lamp_fwd_sm100<128, false><<<grid, block, kSmemLaunch128, stream>>>(P, kmap, vmap, (const uint2*)lut_ptr,
                                                                         (DeviceStats*)stats_ptr);
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
@@ -249,6 +258,7 @@ int lamp_attn_get_stats(lamp_attn_stats* host_out, void* cuda_stream) {
   host_out->exp16_gt1 = ds.v[10];
   host_out->big_rowsum = ds.v[11];
   host_out->device_status = ds.status;
+  for (int i = 0; i < 8; ++i) host_out->phase_cycles[i] = ds.phase[i];
   return ds.status ? LAMP_ERR_DEVICE_TIMEOUT : LAMP_OK;
 }
 

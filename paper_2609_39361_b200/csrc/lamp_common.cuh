@@ -141,7 +141,16 @@ struct DeviceStats {
   unsigned long long v[12];  // active, s1, s2, hist[5], sat8, sat16, gt1, bigrow
   int status;
   int pad;
+  unsigned long long phase[8];  // cycle sums per phase (only with LAMP_PHASE_TIMERS)
 };
+
+#ifdef LAMP_PHASE_TIMERS
+#define LAMP_TIC(var) const long long var = clock64()
+#define LAMP_TOC(slot, var) ph[slot] += clock64() - (var)
+#else
+#define LAMP_TIC(var)
+#define LAMP_TOC(slot, var)
+#endif
 
 __device__ __forceinline__ bool pair_valid(int causal, int window, int i, int j) {
   return (!causal || i <= j) && (window == 0 || j - i < window);

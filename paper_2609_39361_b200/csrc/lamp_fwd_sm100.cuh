@@ -33,8 +33,9 @@ struct Smem {
   static constexpr int kV = kKbf + kTK * D * 2;                   // D/64 boxes [64 keys][64] bf16, SW128
   static constexpr int kPhi = kV + kTK * D * 2;                   // [128][64] bf16, SW128 K-major
   static constexpr int kPlo = kPhi + kBM * kTK * 2;
-  static constexpr int kLut = kPlo + kBM * kTK * 2;               // 256 x u32
-  static constexpr int kBar = kLut + 1024;                        // mbarriers
+  static constexpr int kLut = kPlo + kBM * kTK * 2;               // 128 x uint2
+  static constexpr int kDscr = kLut + 1024;                       // 4 warps x 384 doubles
+  static constexpr int kBar = kDscr + 4 * 384 * 8;                // mbarriers
   static constexpr int kMisc = kBar + 128;                        // tmem slot, lo masks
   static constexpr int kBytes = kMisc + 64;
   static_assert(kKbf % 1024 == 0 && kV % 1024 == 0 && kPhi % 1024 == 0 && kPlo % 1024 == 0, "swizzle atoms");
@@ -97,37 +98,66 @@ __device__ __forceinline__ void chain8(const float* __restrict__ qs, const float
 }
 
 // 16-bit logits of sub-block th for this lane's (quad x 4 keys): a sequential fp64 fma
-// chain over kk, scaled, rounded once to e4m11.
+// chain over kk, scaled, rounded once to e4m11, stored to TMEM columns tdst..tdst+15.
+// The fp32 -> fp64 conversions are the slow
+// part on this GPU, so the warp converts each operand once per 8 channels into a small
+// shared-memory scratch (16 keys and 32 rows as doubles) and every lane reads from there.
+// tq: TMEM columns holding the raw bf16 query row of this lane (row = lane of the group),
+// two channels per column; dscr: 384 doubles per warp.
 template <int D>
-__device__ __forceinline__ void dot16(const float* __restrict__ kf, const __nv_bfloat16* qrow, int64_t qstride,
-                                      int th, int tp, double scale_d, float (&y)[4][4]) {
+__device__ __noinline__ void dot16(const float* __restrict__ kf, uint32_t tq, int th,
+                                   double* dscr, double scale_d, uint32_t tdst) {
+  const int lane = threadIdx.x & 31, qa = lane >> 2, tp = lane & 3;
+  double* kscr = dscr;          // [8 kk][16 keys]
+  double* qscr = dscr + 128;    // [8 kk][32 rows]
   double acc[4][4];
 #pragma unroll
   for (int a = 0; a < 4; ++a)
 #pragma unroll
     for (int b = 0; b < 4; ++b) acc[a][b] = 0.0;
-  const float* kcol = kf + kf_pos(16 * th + 4 * tp);
+  __builtin_assume(__isShared(kf));
+  __builtin_assume(__isShared(dscr));
+  const float* ksrc = kf + qa * kKfStride + kf_pos(16 * th + 4 * tp);   // channel k0 + qa, 4 keys
+  float4 kq = *reinterpret_cast<const float4*>(ksrc);
+  uint4 qraw;
+  ptx::tmem_ld4(tq, qraw);
+  ptx::tmem_wait_ld();
+#pragma unroll 1
   for (int k0 = 0; k0 < D; k0 += 8) {
-    uint4 qraw[4];
-#pragma unroll
-    for (int a = 0; a < 4; ++a) qraw[a] = *reinterpret_cast<const uint4*>(qrow + a * qstride + k0);
+    *reinterpret_cast<double2*>(kscr + qa * 16 + 4 * tp) = make_double2((double)kq.x, (double)kq.y);
+    *reinterpret_cast<double2*>(kscr + qa * 16 + 4 * tp + 2) = make_double2((double)kq.z, (double)kq.w);
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
-      const float4 kq = *reinterpret_cast<const float4*>(kcol + (k0 + e) * kKfStride);
-      const double kd[4] = {(double)kq.x, (double)kq.y, (double)kq.z, (double)kq.w};
-#pragma unroll
-      for (int a = 0; a < 4; ++a) {
-        const uint32_t w = (&qraw[a].x)[e >> 1];
-        const double qd = (double)__uint_as_float((e & 1) ? (w & 0xffff0000u) : (w << 16));
-#pragma unroll
-        for (int b = 0; b < 4; ++b) acc[a][b] = fma(kd[b], qd, acc[a][b]);
-      }
+      const uint32_t w = (&qraw.x)[e >> 1];
+      qscr[e * 32 + lane] = (double)__uint_as_float((e & 1) ? (w & 0xffff0000u) : (w << 16));
     }
+    const int kn = (k0 + 8) & (D - 1);      // next chunk's operands travel while this one is used
+    kq = *reinterpret_cast<const float4*>(ksrc + kn * kKfStride);
+    ptx::tmem_ld4(tq + (kn >> 1), qraw);
+    __syncwarp();
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const double2 k01 = *reinterpret_cast<const double2*>(kscr + e * 16 + 4 * tp);
+      const double2 k23 = *reinterpret_cast<const double2*>(kscr + e * 16 + 4 * tp + 2);
+      const double2 q01 = *reinterpret_cast<const double2*>(qscr + e * 32 + 4 * qa);
+      const double2 q23 = *reinterpret_cast<const double2*>(qscr + e * 32 + 4 * qa + 2);
+      const double kd[4] = {k01.x, k01.y, k23.x, k23.y};
+      const double qd[4] = {q01.x, q01.y, q23.x, q23.y};
+#pragma unroll
+      for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) acc[a][b] = fma(kd[b], qd[a], acc[a][b]);
+    }
+    ptx::tmem_wait_ld();
+    __syncwarp();
   }
+  uint32_t yr[16];
 #pragma unroll
   for (int a = 0; a < 4; ++a)
 #pragma unroll
-    for (int b = 0; b < 4; ++b) y[a][b] = rne_e4m11(__dmul_rn(scale_d, acc[a][b]));
+    for (int b = 0; b < 4; ++b) yr[4 * a + b] = __float_as_uint(rne_e4m11(__dmul_rn(scale_d, acc[a][b])));
+  ptx::tmem_st16(tdst, yr);   // [query a][key b] of the lane's share, parked in its own TMEM lane
+  ptx::tmem_wait_st();
 }
 
 // active, s1, s2, hist, bigrow are warp-uniform; sat8, sat16, gt1 are per-lane partial counts.
@@ -148,17 +178,28 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // Byte address of (row, 16-byte chunk) inside a [rows][64] bf16 tile with the 128-byte swizzle.
 __device__ __forceinline__ uint32_t sw128(int row, int chunk) { return row * 128 + ((chunk ^ (row & 7)) << 4); }
 
+// e8 byte of an 8-bit exponential value (0xF8 = 1.0, E = 0 subnormals in units of 2^-33).
+__device__ __forceinline__ uint32_t enc_exp8(float e) {
+  if (e == 0.0f) return 0u;
+  if (e < 9.313225746154785e-10f) return (uint32_t)(e * 8589934592.0f);
+  return ((__float_as_uint(e) >> 20) & 0x7ffu) - 768u;
+}
+
 // Everything between the low-precision logits and the P V product of Alg. 1 for one
 // (group, key tile): threats and order, stage 1 (eq. (7)), exponentials, lambda / omega,
 // stage 2 (eq. (8)), stage-2 recomputation.  Writes the group's 32 rows of the P tile
 // (bf16 hi, and bf16 lo for 16-bit sub-blocks), returns the flag byte.
+//
+// The 64 first-pass logits of a lane are parked in its own TMEM lane right away (tacc) and
+// read back 16 at a time, so that the per-element work is a short loop instead of a long
+// unrolled stretch of code and the registers are free for the 16-bit path.
 template <int D, bool FULL, bool DUMP>
 __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileGeom& g, float (&acc)[4][16],
-                                              const float* kf, const __nv_bfloat16* qrow, const uint32_t* lut,
-                                              unsigned char* phi, unsigned char* plo, uint32_t tscratch,
-                                              uint32_t& lo_dirty, RowState& st, float (&lam)[4],
-                                              WarpCounters& wc, unsigned long long (&cks)[2], int dump_row0,
-                                              int row0) {
+                                              const float* kf, uint32_t tq, const uint2* lut,
+                                              double* dscr, unsigned char* phi, unsigned char* plo,
+                                              uint32_t tscratch, uint32_t tacc, uint32_t& lo_dirty, RowState& st,
+                                              float (&lam)[4], WarpCounters& wc, unsigned long long (&cks)[2],
+                                              int dump_row0, int row0, long long* ph) {
   const int lane = threadIdx.x & 31;
   const int qa = lane >> 2, th_own = lane & 3;
   const double scale_d = (double)P.scale;
@@ -166,7 +207,7 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
   const bool force8 = P.flags & LAMP_FORCE_8BIT;
   const bool skip1 = (P.flags & (LAMP_FORCE_8BIT | LAMP_NO_STAGE1)) != 0;
 
-  // ---- per sub-block, per query maxima; which sub-blocks are active ----------------------
+  // ---- per sub-block, per query maxima; park the logits; which sub-blocks are active -------
   float cm[4];
 #pragma unroll
   for (int a = 0; a < 4; ++a) {
@@ -175,6 +216,11 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
     for (int b = 0; b < 16; ++b)
       if (vis<FULL>(g, 16 * th_own + b, 4 * qa + a)) m = fmaxf(m, acc[a][b]);
     cm[a] = m;
+    wc.sat8 += m == 448.0f;
+    uint32_t r[16];
+#pragma unroll
+    for (int b = 0; b < 16; ++b) r[b] = __float_as_uint(acc[a][b]);
+    ptx::tmem_st16(tacc + 16 * a, r);
   }
   uint32_t actmask = 0;
 #pragma unroll
@@ -214,6 +260,7 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
 #pragma unroll
   for (int a = 0; a < 4; ++a) muh[a] = st.mu[a];
   uint32_t Theta = 0;
+#pragma unroll 1
   for (int r = 0; r < nact; ++r) {
     const int th = (order >> (2 * r)) & 3;
     bool fail;
@@ -233,27 +280,28 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
     }
     if (!fail) continue;
     Theta |= 1u << th;
-    float y[4][4];
-    dot16<D>(kf, qrow, P.qs[2], th, th_own, scale_d, y);
+    LAMP_TIC(t_d1);
+    dot16<D>(kf, tq, th, dscr, scale_d, tscratch + 16 * th);   // results parked in TMEM
+    LAMP_TOC(4, t_d1);
     uint32_t yr[16];
+    ptx::tmem_ld16(tscratch + 16 * th, yr);
+    ptx::tmem_wait_ld();
 #pragma unroll
     for (int a = 0; a < 4; ++a) {
       float m = -INFINITY;
 #pragma unroll
       for (int b = 0; b < 4; ++b) {
-        yr[4 * a + b] = __float_as_uint(y[a][b]);
+        const float y = __uint_as_float(yr[4 * a + b]);
         if (vis<FULL>(g, 16 * th + 4 * th_own + b, 4 * qa + a)) {
-          m = fmaxf(m, y[a][b]);
-          wc.sat16 += fabsf(y[a][b]) == 448.0f;
+          m = fmaxf(m, y);
+          wc.sat16 += fabsf(y) == 448.0f;
         }
       }
       m = fmaxf(m, __shfl_xor_sync(kFull, m, 1));
       m = fmaxf(m, __shfl_xor_sync(kFull, m, 2));
       muh[a] = fmaxf(muh[a], m);
     }
-    ptx::tmem_st16(tscratch + 16 * th, yr);   // parked in this thread's own TMEM lane
   }
-  if (Theta) ptx::tmem_wait_st();
   if (skip1 && !force16) {
 #pragma unroll
     for (int a = 0; a < 4; ++a) {
@@ -264,98 +312,154 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
     }
   }
 
-  // ---- exponentials: 8-bit through the table, 16-bit correctly rounded -----------------------
+  // ---- exponentials ---------------------------------------------------------------------------
   const bool own_act = (actmask >> th_own) & 1u;
   const bool own8 = own_act && !((Theta >> th_own) & 1u);
-  double rs8[4] = {0.0, 0.0, 0.0, 0.0};
-  if (own_act) {
-#pragma unroll
-    for (int a = 0; a < 4; ++a) {
-      const float m8 = trunc_e4m3(muh[a]);
-#pragma unroll
-      for (int b = 0; b < 16; ++b) {
-        const bool ok = vis<FULL>(g, 16 * th_own + b, 4 * qa + a);
-        float e = 0.0f;
-        if (ok) {
-          const float y8 = acc[a][b];
-          uint32_t eb = 0xffu;
-          wc.sat8 += fabsf(y8) == 448.0f;
-          if (own8) {
-            const uint32_t w = lut[shift_index(__fsub_rn(m8, y8))];
-            e = __uint_as_float(w & 0xffffff00u);
-            eb = w & 0xffu;
-          }
-          if (DUMP) {
-            const uint32_t yb = enc_e4m3(y8);
-            const uint64_t idx = (uint64_t)((16 * th_own + b) * kBQ + 4 * qa + a) << 8;
-            cks[0] += mix64(idx | yb);
-            cks[1] += mix64(idx | eb);
-            if (dump_row0 >= 0) {
-              const size_t off = (size_t)(dump_row0 + 4 * qa + a) * P.seqlen + g.i0 + 16 * th_own + b;
-              if (P.dbg_y8) P.dbg_y8[off] = (uint8_t)yb;
-              if (P.dbg_e8) P.dbg_e8[off] = (uint8_t)eb;
-            }
-          }
-        }
-        acc[a][b] = e;
-        rs8[a] += (double)e;
-      }
-    }
-  } else {
-#pragma unroll
-    for (int a = 0; a < 4; ++a)
-#pragma unroll
-      for (int b = 0; b < 16; ++b) acc[a][b] = 0.0f;
-  }
 
-  // 16-bit exponentials of sub-block th for this lane's (quad x 4 keys); written straight
-  // into the P tile as bf16 hi + lo (12 significant bits = 8 + a remainder of at most 5).
+  // 16-bit: exp of the parked logits of sub-block th for this lane's (quad x 4 keys), written
+  // straight into the P tile as bf16 hi + lo (12 significant bits = 8 + a remainder of <= 5).
   double rs16[4] = {0.0, 0.0, 0.0, 0.0};
-  auto exp_block = [&](int th, const float (&y)[4][4]) {
+  auto exp_block = [&](int th) {
+    uint32_t yr[16];
+    ptx::tmem_ld16(tscratch + 16 * th, yr);
+    ptx::tmem_wait_ld();
+#pragma unroll 1
+    for (int a = 0; a < 4; ++a) {   // one query of the quad per iteration: four independent exps
+      float mh = muh[0];
+      uint32_t y4[4] = {yr[0], yr[1], yr[2], yr[3]};
 #pragma unroll
-    for (int a = 0; a < 4; ++a) {
+      for (int k = 1; k < 4; ++k)
+        if (a == k) {
+          mh = muh[k];
+#pragma unroll
+          for (int b = 0; b < 4; ++b) y4[b] = yr[4 * k + b];
+        }
       float e[4], h[4], l[4];
+      double s = 0.0;
 #pragma unroll
       for (int b = 0; b < 4; ++b) {
         e[b] = 0.0f;
         if (vis<FULL>(g, 16 * th + 4 * th_own + b, 4 * qa + a)) {
-          e[b] = exp16(rne_sig12(__fsub_rn(y[a][b], muh[a])));
+          e[b] = exp16(rne_sig12(__fsub_rn(__uint_as_float(y4[b]), mh)));
           wc.gt1 += e[b] > 1.0f;
         }
-        rs16[a] += (double)e[b];
+        s += (double)e[b];
         h[b] = __bfloat162float(__float2bfloat16_rn(e[b]));
         l[b] = e[b] - h[b];
       }
-      const int row = row0 + 4 * qa + a;
-      const uint32_t off = sw128(row, 2 * th + (th_own >> 1)) + (th_own & 1) * 8;
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        if (a == k) rs16[k] += s;
+      const uint32_t off = sw128(row0 + 4 * qa + a, 2 * th + (th_own >> 1)) + (th_own & 1) * 8;
       *reinterpret_cast<uint2*>(phi + off) = make_uint2(pack_bf16(h[0], h[1]), pack_bf16(h[2], h[3]));
       *reinterpret_cast<uint2*>(plo + off) = make_uint2(pack_bf16(l[0], l[1]), pack_bf16(l[2], l[3]));
     }
   };
-  for (int th = 0; th < 4; ++th) {
-    if (!((Theta >> th) & 1u)) continue;
+  LAMP_TIC(t_e1);
+#pragma unroll 1
+  for (int th = 0; th < 4; ++th)
+    if ((Theta >> th) & 1u) exp_block(th);
+  LAMP_TOC(5, t_e1);
+
+  // 8-bit: through the table, one query row (16 keys) per iteration; the exponentials go
+  // straight to the P tile (4 significant bits: exact in bf16).  Row sums exact in fp32:
+  // entries of 2^-15 or more are multiples of 2^-18 (16 of them stay below 2^5), smaller
+  // ones are multiples of 2^-33 (their sum stays below 2^-11).
+  double rs8[4] = {0.0, 0.0, 0.0, 0.0};
+  ptx::tmem_wait_st();
+#pragma unroll 1
+  for (int a = 0; a < 4; ++a) {
+    const int row = row0 + 4 * qa + a;
+    uint32_t w[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    // (TMEM loads are warp-collective: every lane takes part, whatever its sub-block's path)
     uint32_t yr[16];
-    ptx::tmem_ld16(tscratch + 16 * th, yr);
+    ptx::tmem_ld16(tacc + 16 * a, yr);
     ptx::tmem_wait_ld();
-    float y[4][4];
+    if (own8 || (DUMP && own_act)) {
+      float mh_sel = muh[0];
 #pragma unroll
-    for (int a = 0; a < 4; ++a)
+      for (int k = 1; k < 4; ++k)
+        if (a == k) mh_sel = muh[k];
+      const float m8h = 0.5f * trunc_e4m3(mh_sel);
+      float s_hi = 0.0f, s_lo = 0.0f;
 #pragma unroll
-      for (int b = 0; b < 4; ++b) y[a][b] = __uint_as_float(yr[4 * a + b]);
-    exp_block(th, y);
+      for (int b = 0; b < 16; b += 2) {
+        const bool ok0 = vis<FULL>(g, 16 * th_own + b, 4 * qa + a);
+        const bool ok1 = vis<FULL>(g, 16 * th_own + b + 1, 4 * qa + a);
+        const float y0 = __uint_as_float(yr[b]), y1 = __uint_as_float(yr[b + 1]);
+        float e0 = 0.0f, e1 = 0.0f;
+        if (own8) {
+          // half the shift (exact), rounded to 4 significant bits by the conversion unit: its
+          // e4m3 code indexes the table (shifts below 2^-5 all map to 1.0, as in the 256-entry table)
+          unsigned short pk;
+          asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(pk)
+              : "f"(__fmaf_rn(y1, -0.5f, m8h)), "f"(__fmaf_rn(y0, -0.5f, m8h)));
+          const uint2 w0 = lut[pk & 0x7fu], w1 = lut[(pk >> 8) & 0x7fu];
+          if (ok0) { e0 = __uint_as_float(w0.x); s_lo += __uint_as_float(w0.y); s_hi += e0 - __uint_as_float(w0.y); }
+          if (ok1) { e1 = __uint_as_float(w1.x); s_lo += __uint_as_float(w1.y); s_hi += e1 - __uint_as_float(w1.y); }
+        }
+        w[b >> 1] = pack_bf16(e0, e1);
+        if (DUMP) {
+          const float yy[2] = {y0, y1}, ee[2] = {e0, e1};
+          const bool okk[2] = {ok0, ok1};
+#pragma unroll
+          for (int u = 0; u < 2; ++u) {
+            if (!okk[u]) continue;
+            const uint32_t yb = enc_e4m3(yy[u]);
+            const uint32_t ebb = own8 ? enc_exp8(ee[u]) : 0xffu;
+            const uint64_t idx = (uint64_t)((16 * th_own + b + u) * kBQ + 4 * qa + a) << 8;
+            cks[0] += mix64(idx | yb);
+            cks[1] += mix64(idx | ebb);
+            if (dump_row0 >= 0) {
+              const size_t off = (size_t)(dump_row0 + 4 * qa + a) * P.seqlen + g.i0 + 16 * th_own + b + u;
+              if (P.dbg_y8) P.dbg_y8[off] = (uint8_t)yb;
+              if (P.dbg_e8) P.dbg_e8[off] = (uint8_t)ebb;
+            }
+          }
+        }
+      }
+      const double s = (double)s_hi + (double)s_lo;
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        if (a == k) rs8[k] = s;
+    }
+    if (own8 || !own_act) {   // kept 8-bit values, or the zeros of an inactive sub-block
+      *reinterpret_cast<uint4*>(phi + sw128(row, 2 * th_own)) = make_uint4(w[0], w[1], w[2], w[3]);
+      *reinterpret_cast<uint4*>(phi + sw128(row, 2 * th_own + 1)) = make_uint4(w[4], w[5], w[6], w[7]);
+    }
   }
 
   // ---- lambda_hat (one high-precision exponential per row), omega_hat ------------------------
   double lw[4];
   float omh[4];
   bool big = false;
+  {
+    // one exponential per row: lane theta of the quad takes the quad's query theta
+    float mu_o = st.mu[0], muh_o = muh[0];
+#pragma unroll
+    for (int a = 1; a < 4; ++a)
+      if (th_own == a) { mu_o = st.mu[a]; muh_o = muh[a]; }
+    const float dmu = __fsub_rn(mu_o, muh_o);
+    float l_o = isinf(mu_o) ? 0.0f : 1.0f;
+    if (!isinf(mu_o) && dmu != 0.0f) l_o = (float)exp((double)dmu);
+#pragma unroll
+    for (int a = 0; a < 4; ++a) lam[a] = __shfl_sync(kFull, l_o, (lane & ~3) | a);
+  }
+  double r8free[4];   // this tile's 8-bit mass per row (free sub-blocks only)
 #pragma unroll
   for (int a = 0; a < 4; ++a) {
-    lam[a] = isinf(st.mu[a]) ? 0.0f : (float)exp((double)__fsub_rn(st.mu[a], muh[a]));
     lw[a] = __dmul_rn((double)lam[a], (double)st.om[a]);
-    double R = (own8 ? rs8[a] : 0.0) + rs16[a];
-    R += shfl_xor_d(R, 1);
-    R += shfl_xor_d(R, 2);
+    double R8 = own8 ? rs8[a] : 0.0;
+    R8 += shfl_xor_d(R8, 1);
+    R8 += shfl_xor_d(R8, 2);
+    double R = R8;
+    if (Theta) {
+      double R16 = rs16[a];
+      R16 += shfl_xor_d(R16, 1);
+      R16 += shfl_xor_d(R16, 2);
+      R += R16;
+    }
+    r8free[a] = R8;
     big |= !(R < 4096.0);
     omh[a] = (float)__dadd_rn(lw[a], R);
   }
@@ -363,17 +467,41 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
   // ---- stage 2: block-LAMP problem, eq. (8) -----------------------------------------------------
   const uint32_t freem = actmask & ~Theta;
   uint32_t Rset = 0;
+  LAMP_TIC(t_s2);
+  // Shortcut: sum_i (omega_hat - e_i) e_i <= omega_hat * (8-bit mass), so when that mass is at
+  // most tau * omega_hat (with a margin far above the rounding of the exact evaluation) for
+  // every row, keeping everything is feasible and the exact evaluation would return the empty set.
+  bool need2 = false;
   if (!force8 && !force16 && freem) {
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+      need2 |= !(r8free[a] <= __dmul_rn((double)P.tau * 0.999999998, (double)omh[a]));
+    need2 = __any_sync(kFull, need2);
+  }
+  if (need2) {
     double xi[4] = {0.0, 0.0, 0.0, 0.0};
     if (own8) {
-#pragma unroll
+#pragma unroll 1
       for (int a = 0; a < 4; ++a) {
-        const double oh = (double)omh[a];
+        double oh = (double)omh[0];
+#pragma unroll
+        for (int k = 1; k < 4; ++k)
+          if (a == k) oh = (double)omh[k];
+        // this lane's 16 exponentials of the row, back from the P tile (exact in bf16;
+        // invisible pairs hold 0 and add exactly +0)
+        const int row = row0 + 4 * qa + a;
+        const uint4 p0 = *reinterpret_cast<const uint4*>(phi + sw128(row, 2 * th_own));
+        const uint4 p1 = *reinterpret_cast<const uint4*>(phi + sw128(row, 2 * th_own + 1));
+        const uint32_t pw[8] = {p0.x, p0.y, p0.z, p0.w, p1.x, p1.y, p1.z, p1.w};
+        double x = 0.0;
 #pragma unroll
         for (int b = 0; b < 16; ++b) {
-          const double e = (double)acc[a][b];   // invisible pairs hold 0 and add exactly +0
-          xi[a] = __dadd_rn(xi[a], __dmul_rn(__dsub_rn(oh, e), e));
+          const double e = (double)__uint_as_float((b & 1) ? (pw[b >> 1] & 0xffff0000u) : (pw[b >> 1] << 16));
+          x = __dadd_rn(x, __dmul_rn(__dsub_rn(oh, e), e));
         }
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if (a == k) xi[k] = x;
       }
     }
     uint32_t feas = 0xffffu;
@@ -384,7 +512,7 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
       for (int th = 0; th < 4; ++th) x[th] = shfl_d(xi[a], (lane & ~3) | th);
       const double oh = (double)omh[a];
       const double rhs = __dmul_rn(__dmul_rn((double)P.tau, oh), oh);
-#pragma unroll
+#pragma unroll 1
       for (uint32_t r = 0; r < 16; ++r) {
         const uint32_t keep = freem & ~r;
         double kept = 0.0;
@@ -396,51 +524,53 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
     }
     feas = __reduce_and_sync(kFull, feas);
     int best = 5;   // smallest recompute set, then smallest bitmask, among subsets of the free ones
-#pragma unroll
+#pragma unroll 1
     for (uint32_t r = 0; r < 16; ++r) {
       const int sz = __popc(r);
       if ((r & ~freem) == 0 && ((feas >> r) & 1u) && sz < best) { best = sz; Rset = r; }
     }
   }
+  LAMP_TOC(6, t_s2);
 
   // ---- stage-2 recomputation with the maxima unchanged -------------------------------------------
+#pragma unroll 1
   for (int th = 0; th < 4; ++th) {
     if (!((Rset >> th) & 1u)) continue;
-    float y[4][4];
-    dot16<D>(kf, qrow, P.qs[2], th, th_own, scale_d, y);
+    LAMP_TIC(t_d2);
+    dot16<D>(kf, tq, th, dscr, scale_d, tscratch + 16 * th);
+    LAMP_TOC(4, t_d2);
+    uint32_t yr[16];
+    ptx::tmem_ld16(tscratch + 16 * th, yr);
+    ptx::tmem_wait_ld();
 #pragma unroll
     for (int a = 0; a < 4; ++a)
 #pragma unroll
       for (int b = 0; b < 4; ++b)
-        if (vis<FULL>(g, 16 * th + 4 * th_own + b, 4 * qa + a)) wc.sat16 += fabsf(y[a][b]) == 448.0f;
-    exp_block(th, y);
+        if (vis<FULL>(g, 16 * th + 4 * th_own + b, 4 * qa + a)) wc.sat16 += fabsf(__uint_as_float(yr[4 * a + b])) == 448.0f;
+    LAMP_TIC(t_e2);
+    exp_block(th);
+    LAMP_TOC(5, t_e2);
   }
 
   // ---- state update ------------------------------------------------------------------------------
   const bool keep8 = own8 && !((Rset >> th_own) & 1u);
 #pragma unroll
   for (int a = 0; a < 4; ++a) {
-    double R = (keep8 ? rs8[a] : 0.0) + rs16[a];
-    R += shfl_xor_d(R, 1);
-    R += shfl_xor_d(R, 2);
-    big |= !(R < 4096.0);
     st.mu[a] = muh[a];
-    st.om[a] = (float)__dadd_rn(lw[a], R);
+    st.om[a] = omh[a];          // unchanged unless stage 2 replaced a sub-block
   }
-  // 8-bit exponentials that stay (4 significant bits: exact in bf16) and zeros of inactive
-  // sub-blocks; the lo tile is zero wherever this group has no 16-bit sub-block.
-  const uint32_t hi16 = Theta | Rset;
-  if (keep8 || !own_act) {
+  if (Rset) {
 #pragma unroll
     for (int a = 0; a < 4; ++a) {
-      const int row = row0 + 4 * qa + a;
-      uint32_t w[8];
-#pragma unroll
-      for (int b = 0; b < 8; ++b) w[b] = pack_bf16(acc[a][2 * b], acc[a][2 * b + 1]);
-      *reinterpret_cast<uint4*>(phi + sw128(row, 2 * th_own)) = make_uint4(w[0], w[1], w[2], w[3]);
-      *reinterpret_cast<uint4*>(phi + sw128(row, 2 * th_own + 1)) = make_uint4(w[4], w[5], w[6], w[7]);
+      double R = (keep8 ? rs8[a] : 0.0) + rs16[a];
+      R += shfl_xor_d(R, 1);
+      R += shfl_xor_d(R, 2);
+      big |= !(R < 4096.0);
+      st.om[a] = (float)__dadd_rn(lw[a], R);
     }
   }
+  // the lo tile is zero wherever this group has no 16-bit sub-block
+  const uint32_t hi16 = Theta | Rset;
   if (((lo_dirty & ~hi16) >> th_own) & 1u) {
 #pragma unroll
     for (int a = 0; a < 4; ++a) {
@@ -455,14 +585,19 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
   wc.active += nact;
   wc.s1 += __popc(Theta);
   wc.s2 += __popc(Rset);
-  wc.hist[__popc(hi16)]++;
+  {
+    const int pc = __popc(hi16);
+#pragma unroll
+    for (int i = 0; i < 5; ++i) wc.hist[i] += (pc == i);
+  }
   return Theta | (Rset << 4);
 }
+
 
 template <int D, bool DUMP>
 __global__ void __launch_bounds__(kThreads, 1)
 lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ CUtensorMap kmap,
-               const __grid_constant__ CUtensorMap vmap, const uint32_t* __restrict__ lut_g,
+               const __grid_constant__ CUtensorMap vmap, const uint2* __restrict__ lut_g,
                DeviceStats* __restrict__ gstats) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -473,7 +608,8 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
   unsigned char* vs = smem + L::kV;
   unsigned char* phi = smem + L::kPhi;
   unsigned char* plo = smem + L::kPlo;
-  uint32_t* lut = reinterpret_cast<uint32_t*>(smem + L::kLut);
+  uint2* lut = reinterpret_cast<uint2*>(smem + L::kLut);
+  double* dscr_all = reinterpret_cast<double*>(smem + L::kDscr);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBar);
   uint32_t* tslot = reinterpret_cast<uint32_t*>(smem + L::kMisc);
   uint32_t* lomask = tslot + 1;   // [2]
@@ -506,11 +642,11 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
     lomask[0] = lomask[1] = 0;
   }
   if (warp == kCtrlWarp) {
-    ptx::tmem_alloc(tslot, 256);
+    ptx::tmem_alloc(tslot, 512);
     ptx::tmem_relinquish();
     if (lane == 0) { ptx::prefetch_tensormap(&kmap); ptx::prefetch_tensormap(&vmap); }
   }
-  for (int i = tid; i < 256; i += kThreads) lut[i] = lut_g[i];
+  for (int i = tid; i < 128; i += kThreads) lut[i] = lut_g[i];
   {
     const __nv_bfloat16* qg = P.q + b * P.qs[0] + h * P.qs[1] + (int64_t)m0 * P.qs[2];
     for (int c = tid; c < kBM * D / 8; c += kThreads) {
@@ -620,8 +756,22 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
     const int j0 = m0 + warp * kBQ;
     const int ntk = P.seqlen / kTK;
     const bool dump_rows = DUMP && b == P.dbg_batch && h == P.dbg_head;
-    const __nv_bfloat16* qrow = P.q + b * P.qs[0] + h * P.qs[1] + (int64_t)(j0 + 4 * qa) * P.qs[2];
+    const __nv_bfloat16* qrow = P.q + b * P.qs[0] + h * P.qs[1] + (int64_t)(j0 + lane) * P.qs[2];
+    double* dscr = dscr_all + warp * 384;
     const uint32_t tlane = tbase + ((uint32_t)(warp * 32) << 16);
+    // TMEM columns of this warp's lanes: [0, D) O, [D, D+64) 16-bit logits, [D+64, D+128) parked
+    // first-pass logits, [D+128, D+128+D/2) the lane's raw bf16 query row (for the 16-bit dots)
+#pragma unroll 1
+    for (int c0 = 0; c0 < D / 2; c0 += 16) {
+      uint32_t r[16];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint4 v = *reinterpret_cast<const uint4*>(qrow + 2 * c0 + 8 * i);
+        r[4 * i] = v.x; r[4 * i + 1] = v.y; r[4 * i + 2] = v.z; r[4 * i + 3] = v.w;
+      }
+      ptx::tmem_st16(tlane + D + 128 + c0, r);
+    }
+    ptx::tmem_wait_st();
     RowState st;
 #pragma unroll
     for (int a = 0; a < 4; ++a) { st.mu[a] = -INFINITY; st.om[a] = 0.0f; }
@@ -629,6 +779,8 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
     memset(&wc, 0, sizeof(wc));
     uint32_t lo_dirty = 0;
     bool ok = true;
+    long long ph[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    (void)ph;
 
     for (int n = 0; n < T && ok; ++n) {
       const int t = t_begin + n, i0 = t * kTK;
@@ -641,20 +793,27 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
       uint32_t flag = 0;
       unsigned long long cks[2] = {0ull, 0ull};
 
+      LAMP_TIC(t_w0);
       ok = ptx::mbar_wait(&bars[kKfFull0 + (n & 1)], (n >> 1) & 1, status, kTimeoutCode);
+      LAMP_TOC(0, t_w0);
       float acc[4][16];
+      LAMP_TIC(t_c);
       if (any) chain8<D>(qsT + warp * kBQ + 4 * qa, kf + kf_pos(16 * (lane & 3)), acc);
+      LAMP_TOC(1, t_c);
       // the previous P V product must be complete before O is rescaled or P is overwritten
+      LAMP_TIC(t_w1);
       if (n > 0) ok = ok && ptx::mbar_wait(&bars[kPvDone], (n - 1) & 1, status, kTimeoutCode);
       ptx::tc_fence_after();
+      LAMP_TOC(2, t_w1);
+      LAMP_TIC(t_p);
       if (any) {
         const int dump0 = dump_rows ? j0 : -1;
         if (full)
-          flag = lamp_post<D, true, DUMP>(P, g, acc, kf, qrow, lut, phi, plo, tlane + D, lo_dirty, st, lam, wc,
-                                          cks, dump0, warp * kBQ);
+          flag = lamp_post<D, true, DUMP>(P, g, acc, kf, tlane + D + 128, lut, dscr, phi, plo, tlane + D, tlane + D + 64, lo_dirty, st, lam, wc,
+                                          cks, dump0, warp * kBQ, ph);
         else
-          flag = lamp_post<D, false, DUMP>(P, g, acc, kf, qrow, lut, phi, plo, tlane + D, lo_dirty, st, lam, wc,
-                                           cks, dump0, warp * kBQ);
+          flag = lamp_post<D, false, DUMP>(P, g, acc, kf, tlane + D + 128, lut, dscr, phi, plo, tlane + D, tlane + D + 64, lo_dirty, st, lam, wc,
+                                           cks, dump0, warp * kBQ, ph);
       } else {
         // no visible pair for this group: its rows of the P tile are zero
         for (int c = lane; c < kBQ * 8; c += 32) {
@@ -665,6 +824,8 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
       }
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&bars[kKfEmpty0 + (n & 1)]);
+      LAMP_TOC(3, t_p);
+      LAMP_TIC(t_r);
 
       // O <- diag(lambda_hat) O, only when some row of the group changes its maximum
       bool resc = false;
@@ -694,6 +855,7 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&bars[kPReady]);
+      LAMP_TOC(7, t_r);
 
       const int64_t gt = (((int64_t)b * P.heads_q + h) * (P.seqlen / kBQ) + (j0 / kBQ)) * ntk + t;
       if (lane == 0 && P.flag_mask) P.flag_mask[gt] = (uint8_t)flag;
@@ -757,12 +919,15 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
       atomicAdd(&gstats->v[9], (unsigned long long)sat16);
       atomicAdd(&gstats->v[10], (unsigned long long)gt1);
       atomicAdd(&gstats->v[11], wc.bigrow);
+#ifdef LAMP_PHASE_TIMERS
+      for (int i = 0; i < 8; ++i) atomicAdd(&gstats->phase[i], (unsigned long long)ph[i]);
+#endif
     }
   }
 
   ptx::tc_fence_before();
   __syncthreads();
-  if (warp == kCtrlWarp) ptx::tmem_dealloc(tbase, 256);
+  if (warp == kCtrlWarp) ptx::tmem_dealloc(tbase, 512);
 }
 
 }  // namespace lamp
