@@ -45,7 +45,7 @@ static uint32_t exp8_entry(double s) {
   return (bits & 0xffffff00u) | byte;
 }
 
-constexpr int kSmemLaunch128 = Smem<128>::kBytes + 1024;   // + slack to align the base to 1024 B
+constexpr int kSmemLaunch = SmemLayout::kBytes + 1024;   // + slack to align the base to 1024 B
 
 static thread_local int t_last_cuda = 0;
 static int cuda_fail(cudaError_t e) {
@@ -94,10 +94,12 @@ static int ensure_device(int* dev_out) {
     if (!fn || qr != cudaDriverEntryPointSuccess) return cuda_fail(cudaErrorNotSupported);
     g_encode = (TensorMapEncodeFn)fn;
   }
-  e = cudaFuncSetAttribute(lamp_fwd_sm100<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLaunch128);
-  if (e != cudaSuccess) return cuda_fail(e);
-  e = cudaFuncSetAttribute(lamp_fwd_sm100<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLaunch128);
-  if (e != cudaSuccess) return cuda_fail(e);
+  const void* kernels[4] = {(const void*)lamp_fwd_sm100<128, false>, (const void*)lamp_fwd_sm100<128, true>,
+                            (const void*)lamp_fwd_sm100<256, false>, (const void*)lamp_fwd_sm100<256, true>};
+  for (int i = 0; i < 4; ++i) {
+    e = cudaFuncSetAttribute(kernels[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLaunch);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
   if (dev < 64) g_init.ready[dev] = true;
   return LAMP_OK;
 }
@@ -168,7 +170,7 @@ static int check_params(const void* q, const void* k, const void* v, void* out,
   if ((p->dbg_y8 || p->dbg_e8) &&
       (p->dbg_batch < 0 || p->dbg_batch >= p->batch || p->dbg_head < 0 || p->dbg_head >= p->heads_q))
     return LAMP_ERR_INVALID_ARG;
-  if (p->head_dim != 128) return LAMP_ERR_UNSUPPORTED_SHAPE;
+  if (p->head_dim != 128 && p->head_dim != 256) return LAMP_ERR_UNSUPPORTED_SHAPE;
   if (p->seqlen % kBM) return LAMP_ERR_UNSUPPORTED_SHAPE;
   if (p->batch > 65535 || p->heads_q > 65535) return LAMP_ERR_UNSUPPORTED_SHAPE;
   const int D = p->head_dim;
@@ -229,12 +231,15 @@ int lamp_attn_fwd(const void* q, const void* k, const void* v, void* out, float*
   if (rc) return rc;
   const bool dump = p->dbg_y8 || p->dbg_e8 || p->dbg_checksums;
   dim3 grid(p->seqlen / kBM, p->heads_q, p->batch), block(kThreads);
-  if (dump)
-    lamp_fwd_sm100<128, true><<<grid, block, kSmemLaunch128, stream>>>(P, kmap, vmap, (const uint2*)lut_ptr,
-                                                                       (DeviceStats*)stats_ptr);
-  else
-    lamp_fwd_sm100<128, false><<<grid, block, kSmemLaunch128, stream>>>(P, kmap, vmap, (const uint2*)lut_ptr,
-                                                                        (DeviceStats*)stats_ptr);
+  const uint2* lutp = (const uint2*)lut_ptr;
+  DeviceStats* dsp = (DeviceStats*)stats_ptr;
+  if (p->head_dim == 128) {
+    if (dump) lamp_fwd_sm100<128, true><<<grid, block, kSmemLaunch, stream>>>(P, kmap, vmap, lutp, dsp);
+    else lamp_fwd_sm100<128, false><<<grid, block, kSmemLaunch, stream>>>(P, kmap, vmap, lutp, dsp);
+  } else {
+    if (dump) lamp_fwd_sm100<256, true><<<grid, block, kSmemLaunch, stream>>>(P, kmap, vmap, lutp, dsp);
+    else lamp_fwd_sm100<256, false><<<grid, block, kSmemLaunch, stream>>>(P, kmap, vmap, lutp, dsp);
+  }
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
   return LAMP_OK;

@@ -2,15 +2,23 @@
 //
 // One CTA = 128 query rows of one (batch, query head); key tiles of 64 keys are visited
 // in ascending order (the flags depend on the history of the running maxima, so the key
-// dimension is never split across CTAs).  Seven warps, specialised:
+// dimension is never split across CTAs).  Twelve warps in three groups of four:
 //
-//   warps 0-3  compute: warp w owns the group of 32 rows 32w..32w+31 (and TMEM lanes
-//              32w..32w+31).  Per tile: emulated e4m3 logits on the CUDA cores, stage 1,
-//              exponentials, stage 2, recomputation, rescale of O, P tile to shared memory.
-//   warps 4-5  convert the bf16 K tile that TMA delivered into the fp32, key-contiguous
-//              layout the chain reads (double buffered, one tile ahead of the compute warps).
-//   warp  6    lane 0 issues the TMA loads of K and V and the tcgen05 MMAs O += P V
-//              (bf16 x bf16 -> fp32 in TMEM; 16-bit exponentials enter as bf16 hi + lo).
+//   warps 0-7  compute.  Group g of 32 rows (TMEM lanes 32g..32g+31) is shared by warps g
+//              and g+4, which take the even and the odd key tiles.  The emulated e4m3 chain of
+//              a tile needs nothing from earlier tiles, so while one warp of the pair walks the
+//              (latency-bound, fp64-heavy) decision path of tile n - stage 1, exponentials,
+//              stage 2, recomputation, rescale of O, P tile - the other already runs the chain
+//              of tile n+1 on the same scheduler.  The row state (mu, omega) passes between
+//              them through shared memory, guarded by a token mbarrier.
+//   warps 8-9  convert the bf16 K half-tile (64 keys x 128 channels) that TMA delivered into
+//              the fp32, key-contiguous layout the chain reads (double buffered).
+//   warp  10   issues the TMA loads of K.
+//   warp  11   issues the TMA loads of V and the tcgen05 MMAs O += P V (bf16 x bf16 -> fp32
+//              in TMEM; 16-bit exponentials enter as bf16 hi + lo).
+//
+// head_dim 256 runs as two 128-channel halves per tile: the chain carries its accumulators
+// from the first half to the second, P V is issued per 128 output columns.
 //
 // All hand-offs are mbarriers with bounded waits: a wait that runs out records
 // LAMP_ERR_DEVICE_TIMEOUT and lets the kernel finish instead of hanging the device.
@@ -20,28 +28,37 @@
 
 namespace lamp {
 
-constexpr int kThreads = 224;
-constexpr int kCtrlWarp = 6;
-constexpr int kConvWarps = 2;
+constexpr int kThreads = 384;
+constexpr int kConvWarp0 = 8, kConvWarps = 2, kKWarp = 10, kCtrlWarp = 11;
 constexpr int kTimeoutCode = -4;   // LAMP_ERR_DEVICE_TIMEOUT
+constexpr int kHalf = 128;         // channels per K / V half-tile
 
-template <int D>
-struct Smem {
-  static constexpr int kQs = 0;                                   // [D][128] fp32
-  static constexpr int kKf = kQs + D * kBM * 4;                   // 2 x [D][kKfStride] fp32
-  static constexpr int kKbf = kKf + 2 * D * kKfStride * 4;        // D/64 boxes [64 keys][64] bf16, SW128
-  static constexpr int kV = kKbf + kTK * D * 2;                   // D/64 boxes [64 keys][64] bf16, SW128
-  static constexpr int kPhi = kV + kTK * D * 2;                   // [128][64] bf16, SW128 K-major
+struct SmemLayout {
+  static constexpr int kQs = 0;                                   // head_dim 128: [128][128] fp32 q*scale
+                                                                  // head_dim 256: [256][128] bf16 q
+  static constexpr int kKf = kQs + 65536;                         // 2 x [128][kKfStride] fp32
+  static constexpr int kKbf = kKf + 2 * kHalf * kKfStride * 4;    // 2 boxes [64 keys][64] bf16, SW128
+  static constexpr int kV = kKbf + kTK * kHalf * 2;               // 2 boxes [64 keys][64] bf16, SW128
+  static constexpr int kPhi = kV + kTK * kHalf * 2;               // [128][64] bf16, SW128 K-major
   static constexpr int kPlo = kPhi + kBM * kTK * 2;
   static constexpr int kLut = kPlo + kBM * kTK * 2;               // 128 x uint2
-  static constexpr int kDscr = kLut + 1024;                       // 4 warps x 384 doubles
-  static constexpr int kBar = kDscr + 4 * 384 * 8;                // mbarriers
-  static constexpr int kMisc = kBar + 128;                        // tmem slot, lo masks
+  static constexpr int kDscr = kLut + 1024;                       // 4 groups x 384 doubles
+  static constexpr int kState = kDscr + 4 * 384 * 8;              // mu[128], omega[128], lo_dirty[4]
+  static constexpr int kBar = kState + 1024 + 16;                 // mbarriers
+  static constexpr int kMisc = kBar + 256;                        // tmem slot, lo masks
   static constexpr int kBytes = kMisc + 64;
   static_assert(kKbf % 1024 == 0 && kV % 1024 == 0 && kPhi % 1024 == 0 && kPlo % 1024 == 0, "swizzle atoms");
 };
 
-enum Bar { kKbfFull = 0, kKbfEmpty, kKfFull0, kKfFull1, kKfEmpty0, kKfEmpty1, kVFull, kPReady, kPvDone, kNumBars };
+enum Bar {
+  kKbfFull = 0, kKbfEmpty,
+  // fp32 K half-tile m lives in buffer m & 1 and is announced on barrier m & 3: a compute warp
+  // only meets every other tile, and must never be two completions behind on a barrier it polls
+  kKfFull0, kKfEmpty0 = kKfFull0 + 4, kVFull = kKfEmpty0 + 4, kVHalf, kPReady, kPvDone,
+  kTok0,              // [group][tile parity]: the row state after the previous tile is in shared memory
+  kFin0 = kTok0 + 8,  // [group]: the final row state is in shared memory
+  kNumBars = kFin0 + 4
+};
 
 struct TileGeom {
   int i0, j0, causal, window;
@@ -58,27 +75,44 @@ __device__ __forceinline__ void fma_x2(float& d0, float& d1, float a0, float a1,
 }
 
 // First pass: Y8[i][j] = chain over kk of c <- RNE_e4m3(fma(k, q*scale, c)), c0 = +0
-// (Alg. 1 "accumulate Y in low precision"; Sec. 4.1 round(c + a*b)).  Operands of the next
-// kk are fetched while the current one is processed; FMAs are issued in packed pairs.
-template <int D>
-__device__ __forceinline__ void chain8(const float* __restrict__ qs, const float* __restrict__ kf,
+// (Alg. 1 "accumulate Y in low precision"; Sec. 4.1 round(c + a*b)), 128 channels per call.
+// Operands of the next kk are fetched while the current one is processed; FMAs are issued
+// in packed pairs.  QF32: q holds fp32 q*scale, [kk][128 rows]; else raw bf16 q, scaled here
+// (one fp32 multiply, the same rounding).  FIRST: start from +0, else carry acc on.
+template <bool QF32, bool FIRST>
+__device__ __forceinline__ void chain8(const void* __restrict__ q, const float* __restrict__ kf, float scale,
                                        float (&acc)[4][16]) {
+  if (FIRST) {
 #pragma unroll
-  for (int a = 0; a < 4; ++a)
+    for (int a = 0; a < 4; ++a)
 #pragma unroll
-    for (int b = 0; b < 16; ++b) acc[a][b] = 0.0f;
-  float4 qn = *reinterpret_cast<const float4*>(qs);
+      for (int b = 0; b < 16; ++b) acc[a][b] = 0.0f;
+  }
+  const float* qf = reinterpret_cast<const float*>(q);
+  const __nv_bfloat16* qh = reinterpret_cast<const __nv_bfloat16*>(q);
+  float4 qn = make_float4(0.f, 0.f, 0.f, 0.f);
+  uint2 qnh = make_uint2(0u, 0u);
+  if (QF32) qn = *reinterpret_cast<const float4*>(qf);
+  else qnh = *reinterpret_cast<const uint2*>(qh);
   float4 kn[4];
 #pragma unroll
   for (int c = 0; c < 4; ++c) kn[c] = *reinterpret_cast<const float4*>(kf + 4 * c);
 #pragma unroll 2
-  for (int kk = 0; kk < D; ++kk) {
-    const float q4[4] = {qn.x, qn.y, qn.z, qn.w};
+  for (int kk = 0; kk < kHalf; ++kk) {
+    float q4[4];
+    if (QF32) { q4[0] = qn.x; q4[1] = qn.y; q4[2] = qn.z; q4[3] = qn.w; }
+    else {
+      q4[0] = __fmul_rn(__uint_as_float(qnh.x << 16), scale);
+      q4[1] = __fmul_rn(__uint_as_float(qnh.x & 0xffff0000u), scale);
+      q4[2] = __fmul_rn(__uint_as_float(qnh.y << 16), scale);
+      q4[3] = __fmul_rn(__uint_as_float(qnh.y & 0xffff0000u), scale);
+    }
     float kv[16];
 #pragma unroll
     for (int c = 0; c < 4; ++c) { kv[4 * c] = kn[c].x; kv[4 * c + 1] = kn[c].y; kv[4 * c + 2] = kn[c].z; kv[4 * c + 3] = kn[c].w; }
-    const int nx = (kk + 1) & (D - 1);
-    qn = *reinterpret_cast<const float4*>(qs + nx * kBM);
+    const int nx = (kk + 1) & (kHalf - 1);
+    if (QF32) qn = *reinterpret_cast<const float4*>(qf + nx * kBM);
+    else qnh = *reinterpret_cast<const uint2*>(qh + nx * kBM);
 #pragma unroll
     for (int c = 0; c < 4; ++c) kn[c] = *reinterpret_cast<const float4*>(kf + nx * kKfStride + 4 * c);
 #pragma unroll
@@ -97,17 +131,20 @@ __device__ __forceinline__ void chain8(const float* __restrict__ qs, const float
   }
 }
 
-// 16-bit logits of sub-block th for this lane's (quad x 4 keys): a sequential fp64 fma
+// 16-bit logits of one sub-block for this lane's (quad x 4 keys): a sequential fp64 fma
 // chain over kk, scaled, rounded once to e4m11, stored to TMEM columns tdst..tdst+15.
-// The fp32 -> fp64 conversions are the slow
-// part on this GPU, so the warp converts each operand once per 8 channels into a small
-// shared-memory scratch (16 keys and 32 rows as doubles) and every lane reads from there.
-// tq: TMEM columns holding the raw bf16 query row of this lane (row = lane of the group),
-// two channels per column; dscr: 384 doubles per warp.
+// The fp32 -> fp64 conversions are the slow part on this GPU, so the warp converts each
+// operand once per 8 channels into a small shared-memory scratch (16 keys and 32 rows as
+// doubles) and every lane reads from there.
+// krow: global bf16 row of the sub-block's first key (lanes 0-15 fetch key `lane`, 16 bytes
+// per 8 channels; the rows were just streamed through L2 by TMA); tq: TMEM columns holding
+// the raw bf16 query row of this lane (row = lane of the group), two channels per column;
+// dscr: 384 doubles for the warp.
 template <int D>
-__device__ __noinline__ void dot16(const float* __restrict__ kf, uint32_t tq, int th,
+__device__ __noinline__ void dot16(const __nv_bfloat16* __restrict__ krow, int64_t kstride, uint32_t tq,
                                    double* dscr, double scale_d, uint32_t tdst) {
   const int lane = threadIdx.x & 31, qa = lane >> 2, tp = lane & 3;
+  __builtin_assume(__isShared(dscr));
   double* kscr = dscr;          // [8 kk][16 keys]
   double* qscr = dscr + 128;    // [8 kk][32 rows]
   double acc[4][4];
@@ -115,24 +152,24 @@ __device__ __noinline__ void dot16(const float* __restrict__ kf, uint32_t tq, in
   for (int a = 0; a < 4; ++a)
 #pragma unroll
     for (int b = 0; b < 4; ++b) acc[a][b] = 0.0;
-  __builtin_assume(__isShared(kf));
-  __builtin_assume(__isShared(dscr));
-  const float* ksrc = kf + qa * kKfStride + kf_pos(16 * th + 4 * tp);   // channel k0 + qa, 4 keys
-  float4 kq = *reinterpret_cast<const float4*>(ksrc);
+  const __nv_bfloat16* ksrc = krow + (int64_t)(lane & 15) * kstride;
+  uint4 kraw = *reinterpret_cast<const uint4*>(ksrc);
   uint4 qraw;
   ptx::tmem_ld4(tq, qraw);
   ptx::tmem_wait_ld();
 #pragma unroll 1
   for (int k0 = 0; k0 < D; k0 += 8) {
-    *reinterpret_cast<double2*>(kscr + qa * 16 + 4 * tp) = make_double2((double)kq.x, (double)kq.y);
-    *reinterpret_cast<double2*>(kscr + qa * 16 + 4 * tp + 2) = make_double2((double)kq.z, (double)kq.w);
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
-      const uint32_t w = (&qraw.x)[e >> 1];
-      qscr[e * 32 + lane] = (double)__uint_as_float((e & 1) ? (w & 0xffff0000u) : (w << 16));
+      const uint32_t wq = (&qraw.x)[e >> 1];
+      qscr[e * 32 + lane] = (double)__uint_as_float((e & 1) ? (wq & 0xffff0000u) : (wq << 16));
+      if (lane < 16) {
+        const uint32_t wk = (&kraw.x)[e >> 1];
+        kscr[e * 16 + lane] = (double)__uint_as_float((e & 1) ? (wk & 0xffff0000u) : (wk << 16));
+      }
     }
     const int kn = (k0 + 8) & (D - 1);      // next chunk's operands travel while this one is used
-    kq = *reinterpret_cast<const float4*>(ksrc + kn * kKfStride);
+    kraw = *reinterpret_cast<const uint4*>(ksrc + kn);
     ptx::tmem_ld4(tq + (kn >> 1), qraw);
     __syncwarp();
 #pragma unroll
@@ -195,8 +232,8 @@ __device__ __forceinline__ uint32_t enc_exp8(float e) {
 // unrolled stretch of code and the registers are free for the 16-bit path.
 template <int D, bool FULL, bool DUMP>
 __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileGeom& g, float (&acc)[4][16],
-                                              const float* kf, uint32_t tq, const uint2* lut,
-                                              double* dscr, unsigned char* phi, unsigned char* plo,
+                                              const __nv_bfloat16* ktile, int64_t kstride, uint32_t tq,
+                                              const uint2* lut, double* dscr, unsigned char* phi, unsigned char* plo,
                                               uint32_t tscratch, uint32_t tacc, uint32_t& lo_dirty, RowState& st,
                                               float (&lam)[4], WarpCounters& wc, unsigned long long (&cks)[2],
                                               int dump_row0, int row0, long long* ph) {
@@ -281,7 +318,7 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
     if (!fail) continue;
     Theta |= 1u << th;
     LAMP_TIC(t_d1);
-    dot16<D>(kf, tq, th, dscr, scale_d, tscratch + 16 * th);   // results parked in TMEM
+    dot16<D>(ktile + (int64_t)(16 * th) * kstride, kstride, tq, dscr, scale_d, tscratch + 16 * th);   // results parked in TMEM
     LAMP_TOC(4, t_d1);
     uint32_t yr[16];
     ptx::tmem_ld16(tscratch + 16 * th, yr);
@@ -537,7 +574,7 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
   for (int th = 0; th < 4; ++th) {
     if (!((Rset >> th) & 1u)) continue;
     LAMP_TIC(t_d2);
-    dot16<D>(kf, tq, th, dscr, scale_d, tscratch + 16 * th);
+    dot16<D>(ktile + (int64_t)(16 * th) * kstride, kstride, tq, dscr, scale_d, tscratch + 16 * th);
     LAMP_TOC(4, t_d2);
     uint32_t yr[16];
     ptx::tmem_ld16(tscratch + 16 * th, yr);
@@ -599,10 +636,13 @@ __global__ void __launch_bounds__(kThreads, 1)
 lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ CUtensorMap kmap,
                const __grid_constant__ CUtensorMap vmap, const uint2* __restrict__ lut_g,
                DeviceStats* __restrict__ gstats) {
+  static_assert(D == 128 || D == 256, "head_dim");
+  constexpr int NH = D / kHalf;          // 128-channel halves per tile
+  constexpr bool QF32 = (D == 128);      // Q operand of the chain: fp32 q*scale, or raw bf16
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
-  using L = Smem<D>;
-  float* qsT = reinterpret_cast<float*>(smem + L::kQs);
+  using L = SmemLayout;
+  unsigned char* qs = smem + L::kQs;
   float* kf_all = reinterpret_cast<float*>(smem + L::kKf);
   unsigned char* kbf = smem + L::kKbf;
   unsigned char* vs = smem + L::kV;
@@ -610,6 +650,9 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
   unsigned char* plo = smem + L::kPlo;
   uint2* lut = reinterpret_cast<uint2*>(smem + L::kLut);
   double* dscr_all = reinterpret_cast<double*>(smem + L::kDscr);
+  float* st_mu = reinterpret_cast<float*>(smem + L::kState);
+  float* st_om = st_mu + kBM;
+  uint32_t* st_lod = reinterpret_cast<uint32_t*>(st_om + kBM);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBar);
   uint32_t* tslot = reinterpret_cast<uint32_t*>(smem + L::kMisc);
   uint32_t* lomask = tslot + 1;   // [2]
@@ -626,18 +669,22 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
   if (P.causal) t_end = min(t_end, (m0 + kBM - 1) / kTK + 1);
   if (P.window > 0) t_begin = max(0, m0 - P.window + 1) / kTK;
   const int T = t_end - t_begin;
+  const int M = T * NH;                       // half-tiles of the K (and V) stream
+  constexpr uint32_t kHalfBytes = kTK * kHalf * 2;
 
   // ---- set-up ---------------------------------------------------------------------------------
   if (tid == 0) {
     ptx::mbar_init(&bars[kKbfFull], 1);
     ptx::mbar_init(&bars[kKbfEmpty], kConvWarps);
-    ptx::mbar_init(&bars[kKfFull0], kConvWarps);
-    ptx::mbar_init(&bars[kKfFull1], kConvWarps);
-    ptx::mbar_init(&bars[kKfEmpty0], 4);
-    ptx::mbar_init(&bars[kKfEmpty1], 4);
+    for (int i = 0; i < 4; ++i) {
+      ptx::mbar_init(&bars[kKfFull0 + i], kConvWarps);
+      ptx::mbar_init(&bars[kKfEmpty0 + i], 4);
+    }
     ptx::mbar_init(&bars[kVFull], 1);
+    ptx::mbar_init(&bars[kVHalf], 1);
     ptx::mbar_init(&bars[kPReady], 4);
     ptx::mbar_init(&bars[kPvDone], 1);
+    for (int i = 0; i < 12; ++i) ptx::mbar_init(&bars[kTok0 + i], 1);
     ptx::fence_barrier_init();
     lomask[0] = lomask[1] = 0;
   }
@@ -655,14 +702,20 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
         const uint32_t w = (&raw.x)[e >> 1];
-        const float f = __uint_as_float((e & 1) ? (w & 0xffff0000u) : (w << 16));
-        qsT[(k0 + e) * kBM + row] = __fmul_rn(f, P.scale);
+        if (QF32) {
+          const float f = __uint_as_float((e & 1) ? (w & 0xffff0000u) : (w << 16));
+          reinterpret_cast<float*>(qs)[(k0 + e) * kBM + row] = __fmul_rn(f, P.scale);
+        } else {
+          reinterpret_cast<unsigned short*>(qs)[(k0 + e) * kBM + row] = (unsigned short)((e & 1) ? (w >> 16) : (w & 0xffffu));
+        }
       }
     }
     for (int c = tid; c < kBM * kTK * 2 / 16; c += kThreads) {
       reinterpret_cast<uint4*>(phi)[c] = make_uint4(0, 0, 0, 0);
       reinterpret_cast<uint4*>(plo)[c] = make_uint4(0, 0, 0, 0);
     }
+    for (int c = tid; c < kBM; c += kThreads) { st_mu[c] = -INFINITY; st_om[c] = 0.0f; }
+    if (tid < 4) st_lod[tid] = 0;
   }
   ptx::fence_proxy_async();
   ptx::tc_fence_before();
@@ -670,121 +723,131 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
   ptx::tc_fence_after();
   const uint32_t tbase = *tslot;
 
-  if (warp == kCtrlWarp) {
-    // =========================== control: TMA loads and MMA issue ================================
-    // (all 32 lanes walk the loop so that the warp stays converged; lane 0 issues)
-    constexpr uint32_t kTileBytes = kTK * D * 2;
-    constexpr uint32_t idesc = ptx::idesc_bf16(kBM, D, 1);
-    bool ok = true;
-    if (lane == 0) {
-      ptx::mbar_arrive_expect_tx(&bars[kKbfFull], kTileBytes);
-      ptx::mbar_arrive_expect_tx(&bars[kVFull], kTileBytes);
-#pragma unroll
-      for (int x = 0; x < D / 64; ++x) {
-        ptx::tma_load_4d(kbf + x * 8192, &kmap, &bars[kKbfFull], 64 * x, t_begin * kTK, hk, b);
-        ptx::tma_load_4d(vs + x * 8192, &vmap, &bars[kVFull], 64 * x, t_begin * kTK, hk, b);
-      }
-    }
-    __syncwarp();
-    for (int n = 0; n < T && ok; ++n) {
-      if (n + 1 < T) {
-        ok = ptx::mbar_wait(&bars[kKbfEmpty], n & 1, status, kTimeoutCode);
+  if (warp >= 8) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+    if (warp == kKWarp) {
+      // =========================== K stream: one TMA half-tile ahead of the converters ===========
+      // (all 32 lanes walk the loop so that the warp stays converged; lane 0 issues)
+      bool ok = true;
+      for (int m = 0; m < M && ok; ++m) {
+        if (m > 0) ok = ptx::mbar_wait(&bars[kKbfEmpty], (m - 1) & 1, status, kTimeoutCode);
         if (lane == 0 && ok) {
-          ptx::mbar_arrive_expect_tx(&bars[kKbfFull], kTileBytes);
+          ptx::mbar_arrive_expect_tx(&bars[kKbfFull], kHalfBytes);
 #pragma unroll
-          for (int x = 0; x < D / 64; ++x)
-            ptx::tma_load_4d(kbf + x * 8192, &kmap, &bars[kKbfFull], 64 * x, (t_begin + n + 1) * kTK, hk, b);
+          for (int x = 0; x < 2; ++x)
+            ptx::tma_load_4d(kbf + x * 8192, &kmap, &bars[kKbfFull], kHalf * (m % NH) + 64 * x,
+                             (t_begin + m / NH) * kTK, hk, b);
         }
+        ok = __all_sync(kFull, ok);
       }
-      ok = ok && ptx::mbar_wait(&bars[kPReady], n & 1, status, kTimeoutCode);
-      ok = ok && ptx::mbar_wait(&bars[kVFull], n & 1, status, kTimeoutCode);
-      ok = __all_sync(kFull, ok);
-      ptx::tc_fence_after();
-      if (lane == 0 && ok) {
-        const uint32_t lom = lomask[n & 1];
-        lomask[n & 1] = 0;
+    } else if (warp == kCtrlWarp) {
+      // =========================== V stream and the MMAs O += P V ====================================
+      constexpr uint32_t idesc = ptx::idesc_bf16(kBM, kHalf, 1);
+      bool ok = true;
+      auto load_v = [&](int mv) {
+        ptx::mbar_arrive_expect_tx(&bars[kVFull], kHalfBytes);
 #pragma unroll
-        for (int ks = 0; ks < 4; ++ks) {
-          const uint64_t bd = ptx::smem_desc_sw128(ptx::smem_u32(vs) + ks * 2048, 8192, 1024);
-          ptx::umma_bf16(tbase, ptx::smem_desc_sw128(ptx::smem_u32(phi) + ks * 32, 16, 1024), bd, idesc,
-                         (n > 0 || ks > 0) ? 1u : 0u);
-          if ((lom >> ks) & 1u)
-            ptx::umma_bf16(tbase, ptx::smem_desc_sw128(ptx::smem_u32(plo) + ks * 32, 16, 1024), bd, idesc, 1u);
-        }
-        ptx::umma_commit(&bars[kPvDone]);
-      }
+        for (int x = 0; x < 2; ++x)
+          ptx::tma_load_4d(vs + x * 8192, &vmap, &bars[kVFull], kHalf * (mv % NH) + 64 * x,
+                           (t_begin + mv / NH) * kTK, hk, b);
+      };
+      if (lane == 0) load_v(0);
       __syncwarp();
-      if (n + 1 < T && ok) {
-        ok = ptx::mbar_wait(&bars[kPvDone], n & 1, status, kTimeoutCode);
-        if (lane == 0 && ok) {
-          ptx::mbar_arrive_expect_tx(&bars[kVFull], kTileBytes);
+      for (int n = 0; n < T && ok; ++n) {
+        ok = ptx::mbar_wait(&bars[kPReady], n & 1, status, kTimeoutCode);
+        uint32_t lom = 0;
+#pragma unroll 1
+        for (int hh = 0; hh < NH && ok; ++hh) {
+          const int mv = n * NH + hh;
+          ok = ptx::mbar_wait(&bars[kVFull], mv & 1, status, kTimeoutCode);
+          ok = __all_sync(kFull, ok);
+          ptx::tc_fence_after();
+          if (lane == 0 && ok) {
+            if (hh == 0) { lom = lomask[n & 1]; lomask[n & 1] = 0; }
 #pragma unroll
-          for (int x = 0; x < D / 64; ++x)
-            ptx::tma_load_4d(vs + x * 8192, &vmap, &bars[kVFull], 64 * x, (t_begin + n + 1) * kTK, hk, b);
+            for (int ks = 0; ks < 4; ++ks) {
+              const uint64_t bd = ptx::smem_desc_sw128(ptx::smem_u32(vs) + ks * 2048, 8192, 1024);
+              ptx::umma_bf16(tbase + kHalf * hh, ptx::smem_desc_sw128(ptx::smem_u32(phi) + ks * 32, 16, 1024), bd,
+                             idesc, (n > 0 || ks > 0) ? 1u : 0u);
+              if ((lom >> ks) & 1u)
+                ptx::umma_bf16(tbase + kHalf * hh, ptx::smem_desc_sw128(ptx::smem_u32(plo) + ks * 32, 16, 1024), bd,
+                               idesc, 1u);
+            }
+            ptx::umma_commit(hh + 1 < NH ? &bars[kVHalf] : &bars[kPvDone]);
+          }
+          __syncwarp();
+          // the V buffer is single: the next half-tile may land once these MMAs have read it
+          if (mv + 1 < M && ok) {
+            ok = ptx::mbar_wait(hh + 1 < NH ? &bars[kVHalf] : &bars[kPvDone], n & 1, status, kTimeoutCode);
+            if (lane == 0 && ok) load_v(mv + 1);
+          }
+          ok = __all_sync(kFull, ok);
         }
       }
-      ok = __all_sync(kFull, ok);
-    }
-  } else if (warp >= 4) {
-    // =========================== converters: bf16 K tile -> fp32, key-contiguous ===================
-    const int key = tid - 128;         // 0..63: one key of the tile per thread
-    bool ok = true;
-    for (int n = 0; n < T && ok; ++n) {
-      float* kf = kf_all + (n & 1) * D * kKfStride;
-      ok = ptx::mbar_wait(&bars[kKbfFull], n & 1, status, kTimeoutCode);
-      if (n >= 2) ok = ok && ptx::mbar_wait(&bars[kKfEmpty0 + (n & 1)], ((n >> 1) - 1) & 1, status, kTimeoutCode);
+    } else if (warp < kConvWarp0 + kConvWarps) {
+      // =========================== converters: bf16 K half-tile -> fp32, key-contiguous ==============
+      const int key = tid - kConvWarp0 * 32;   // 0..63: one key of the tile per thread
       const int pos = kf_pos(key);
+      bool ok = true;
+      for (int m = 0; m < M && ok; ++m) {
+        float* kf = kf_all + (m & 1) * kHalf * kKfStride;
+        ok = ptx::mbar_wait(&bars[kKbfFull], m & 1, status, kTimeoutCode);
+        if (m >= 2) ok = ok && ptx::mbar_wait(&bars[kKfEmpty0 + ((m - 2) & 3)], ((m - 2) >> 2) & 1, status, kTimeoutCode);
 #pragma unroll 4
-      for (int c = 0; c < D / 8; ++c) {   // 16-byte chunk c: channels 8c..8c+7 of this key
-        const int box = c >> 3, cc = c & 7;
-        const uint4 raw = *reinterpret_cast<const uint4*>(kbf + box * 8192 + sw128(key, cc));
+        for (int c = 0; c < kHalf / 8; ++c) {   // 16-byte chunk c: channels 8c..8c+7 of this key
+          const uint4 raw = *reinterpret_cast<const uint4*>(kbf + (c >> 3) * 8192 + sw128(key, c & 7));
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const uint32_t w = (&raw.x)[e >> 1];
-          kf[(8 * c + e) * kKfStride + pos] = __uint_as_float((e & 1) ? (w & 0xffff0000u) : (w << 16));
+          for (int e = 0; e < 8; ++e) {
+            const uint32_t w = (&raw.x)[e >> 1];
+            kf[(8 * c + e) * kKfStride + pos] = __uint_as_float((e & 1) ? (w & 0xffff0000u) : (w << 16));
+          }
         }
-      }
-      __syncwarp();
-      if (lane == 0) {
-        ptx::mbar_arrive(&bars[kKfFull0 + (n & 1)]);
-        ptx::mbar_arrive(&bars[kKbfEmpty]);
+        __syncwarp();
+        if (lane == 0) {
+          ptx::mbar_arrive(&bars[kKfFull0 + (m & 3)]);
+          ptx::mbar_arrive(&bars[kKbfEmpty]);
+        }
       }
     }
   } else {
-    // =========================== compute: one group of 32 query rows per warp =====================
+    // =========================== compute: two warps per group of 32 query rows =====================
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+    const int grp = warp & 3, side = warp >> 2;   // side 0 takes the even tiles, side 1 the odd ones
     const int qa = lane >> 2;
-    const int j0 = m0 + warp * kBQ;
+    const int j0 = m0 + grp * kBQ;
     const int ntk = P.seqlen / kTK;
     const bool dump_rows = DUMP && b == P.dbg_batch && h == P.dbg_head;
-    const __nv_bfloat16* qrow = P.q + b * P.qs[0] + h * P.qs[1] + (int64_t)(j0 + lane) * P.qs[2];
-    double* dscr = dscr_all + warp * 384;
-    const uint32_t tlane = tbase + ((uint32_t)(warp * 32) << 16);
-    // TMEM columns of this warp's lanes: [0, D) O, [D, D+64) 16-bit logits, [D+64, D+128) parked
-    // first-pass logits, [D+128, D+128+D/2) the lane's raw bf16 query row (for the 16-bit dots)
+    const __nv_bfloat16* kg = P.k + b * P.ks[0] + hk * P.ks[1];
+    double* dscr = dscr_all + grp * 384;
+    const uint32_t tlane = tbase + ((uint32_t)(grp * 32) << 16);
+    // TMEM columns of the group's lanes: [0, D) O, then 64 for the 16-bit logits, 64 for the parked
+    // first-pass logits, D/2 for the lane's raw bf16 query row (operand of the 16-bit dots)
+    const uint32_t tscr = tlane + D, tacc = tlane + D + 64, tq = tlane + D + 128;
+    if (side == 0) {
+      const __nv_bfloat16* qrow = P.q + b * P.qs[0] + h * P.qs[1] + (int64_t)(j0 + lane) * P.qs[2];
 #pragma unroll 1
-    for (int c0 = 0; c0 < D / 2; c0 += 16) {
-      uint32_t r[16];
+      for (int c0 = 0; c0 < D / 2; c0 += 16) {
+        uint32_t r[16];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const uint4 v = *reinterpret_cast<const uint4*>(qrow + 2 * c0 + 8 * i);
-        r[4 * i] = v.x; r[4 * i + 1] = v.y; r[4 * i + 2] = v.z; r[4 * i + 3] = v.w;
+        for (int i = 0; i < 4; ++i) {
+          const uint4 v = *reinterpret_cast<const uint4*>(qrow + 2 * c0 + 8 * i);
+          r[4 * i] = v.x; r[4 * i + 1] = v.y; r[4 * i + 2] = v.z; r[4 * i + 3] = v.w;
+        }
+        ptx::tmem_st16(tq + c0, r);
       }
-      ptx::tmem_st16(tlane + D + 128 + c0, r);
+      ptx::tmem_wait_st();
     }
-    ptx::tmem_wait_st();
     RowState st;
-#pragma unroll
-    for (int a = 0; a < 4; ++a) { st.mu[a] = -INFINITY; st.om[a] = 0.0f; }
     WarpCounters wc;
     memset(&wc, 0, sizeof(wc));
     uint32_t lo_dirty = 0;
     bool ok = true;
     long long ph[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     (void)ph;
+    const unsigned char* q_quad = qs + (QF32 ? 4 : 2) * (grp * kBQ + 4 * qa);
 
-    for (int n = 0; n < T && ok; ++n) {
+    for (int n = side; n < T && ok; n += 2) {
       const int t = t_begin + n, i0 = t * kTK;
-      const float* kf = kf_all + (n & 1) * D * kKfStride;
       TileGeom g;
       g.i0 = i0; g.j0 = j0; g.causal = P.causal; g.window = P.window;
       const bool any = (!P.causal || i0 <= j0 + 31) && (P.window == 0 || j0 - (i0 + 63) < P.window);
@@ -793,38 +856,69 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
       uint32_t flag = 0;
       unsigned long long cks[2] = {0ull, 0ull};
 
-      LAMP_TIC(t_w0);
-      ok = ptx::mbar_wait(&bars[kKfFull0 + (n & 1)], (n >> 1) & 1, status, kTimeoutCode);
-      LAMP_TOC(0, t_w0);
+      // ---- emulated 8-bit logits: needs only K and Q, runs ahead of the other warp's decision path
       float acc[4][16];
-      LAMP_TIC(t_c);
-      if (any) chain8<D>(qsT + warp * kBQ + 4 * qa, kf + kf_pos(16 * (lane & 3)), acc);
-      LAMP_TOC(1, t_c);
-      // the previous P V product must be complete before O is rescaled or P is overwritten
+#pragma unroll
+      for (int hh = 0; hh < NH; ++hh) {
+        const int m = n * NH + hh;
+        const float* kf = kf_all + (m & 1) * kHalf * kKfStride + kf_pos(16 * (lane & 3));
+        LAMP_TIC(t_w0);
+        ok = ok && ptx::mbar_wait(&bars[kKfFull0 + (m & 3)], (m >> 2) & 1, status, kTimeoutCode);
+        LAMP_TOC(0, t_w0);
+        LAMP_TIC(t_c);
+        if (any) {
+          const unsigned char* qh = q_quad + (size_t)hh * kHalf * kBM * (QF32 ? 4 : 2);
+          if (hh == 0) chain8<QF32, true>(qh, kf, P.scale, acc);
+          else chain8<QF32, false>(qh, kf, P.scale, acc);
+        }
+        LAMP_TOC(1, t_c);
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&bars[kKfEmpty0 + (m & 3)]);
+      }
+
+      // ---- the row state after tile n-1 (from the other warp), and O / P free again ---------------
       LAMP_TIC(t_w1);
-      if (n > 0) ok = ok && ptx::mbar_wait(&bars[kPvDone], (n - 1) & 1, status, kTimeoutCode);
+      if (n > 0) {
+        ok = ok && ptx::mbar_wait(&bars[kTok0 + 2 * grp + (n & 1)], (((n + 1) >> 1) - 1) & 1, status, kTimeoutCode);
+        ok = ok && ptx::mbar_wait(&bars[kPvDone], (n - 1) & 1, status, kTimeoutCode);
+      }
       ptx::tc_fence_after();
+      {
+        const float4 m4 = *reinterpret_cast<const float4*>(st_mu + grp * kBQ + 4 * qa);
+        const float4 o4 = *reinterpret_cast<const float4*>(st_om + grp * kBQ + 4 * qa);
+        st.mu[0] = m4.x; st.mu[1] = m4.y; st.mu[2] = m4.z; st.mu[3] = m4.w;
+        st.om[0] = o4.x; st.om[1] = o4.y; st.om[2] = o4.z; st.om[3] = o4.w;
+        lo_dirty = st_lod[grp];
+      }
       LAMP_TOC(2, t_w1);
       LAMP_TIC(t_p);
       if (any) {
         const int dump0 = dump_rows ? j0 : -1;
+        const __nv_bfloat16* ktile = kg + (int64_t)i0 * P.ks[2];
         if (full)
-          flag = lamp_post<D, true, DUMP>(P, g, acc, kf, tlane + D + 128, lut, dscr, phi, plo, tlane + D, tlane + D + 64, lo_dirty, st, lam, wc,
-                                          cks, dump0, warp * kBQ, ph);
+          flag = lamp_post<D, true, DUMP>(P, g, acc, ktile, P.ks[2], tq, lut, dscr, phi, plo, tscr, tacc, lo_dirty,
+                                          st, lam, wc, cks, dump0, grp * kBQ, ph);
         else
-          flag = lamp_post<D, false, DUMP>(P, g, acc, kf, tlane + D + 128, lut, dscr, phi, plo, tlane + D, tlane + D + 64, lo_dirty, st, lam, wc,
-                                           cks, dump0, warp * kBQ, ph);
+          flag = lamp_post<D, false, DUMP>(P, g, acc, ktile, P.ks[2], tq, lut, dscr, phi, plo, tscr, tacc, lo_dirty,
+                                           st, lam, wc, cks, dump0, grp * kBQ, ph);
+        if ((lane & 3) == 0) {
+          *reinterpret_cast<float4*>(st_mu + grp * kBQ + 4 * qa) = make_float4(st.mu[0], st.mu[1], st.mu[2], st.mu[3]);
+          *reinterpret_cast<float4*>(st_om + grp * kBQ + 4 * qa) = make_float4(st.om[0], st.om[1], st.om[2], st.om[3]);
+        }
       } else {
         // no visible pair for this group: its rows of the P tile are zero
         for (int c = lane; c < kBQ * 8; c += 32) {
-          *reinterpret_cast<uint4*>(phi + sw128(warp * kBQ + (c >> 3), c & 7)) = make_uint4(0, 0, 0, 0);
-          if (lo_dirty) *reinterpret_cast<uint4*>(plo + sw128(warp * kBQ + (c >> 3), c & 7)) = make_uint4(0, 0, 0, 0);
+          *reinterpret_cast<uint4*>(phi + sw128(grp * kBQ + (c >> 3), c & 7)) = make_uint4(0, 0, 0, 0);
+          if (lo_dirty) *reinterpret_cast<uint4*>(plo + sw128(grp * kBQ + (c >> 3), c & 7)) = make_uint4(0, 0, 0, 0);
         }
         lo_dirty = 0;
       }
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(&bars[kKfEmpty0 + (n & 1)]);
+      if (lane == 0) st_lod[grp] = lo_dirty;
       LAMP_TOC(3, t_p);
+      // hand the state (and the TMEM scratch columns) to the other warp of the pair
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(n + 1 < T ? &bars[kTok0 + 2 * grp + ((n + 1) & 1)] : &bars[kFin0 + grp]);
       LAMP_TIC(t_r);
 
       // O <- diag(lambda_hat) O, only when some row of the group changes its maximum
@@ -832,12 +926,10 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
 #pragma unroll
       for (int a = 0; a < 4; ++a) resc |= lam[a] != 1.0f;
       if (n > 0 && __any_sync(kFull, resc)) {
-        float lrow = 1.0f;   // lambda of the row this lane owns in TMEM (row = lane)
+        float lrow = lam[0];   // lambda of the row this lane owns in TMEM (row = lane = 4*qa + (lane & 3))
 #pragma unroll
-        for (int a = 0; a < 4; ++a) {
-          const float v = __shfl_sync(kFull, lam[a], (lane >> 2) << 2);
-          if ((lane & 3) == a) lrow = v;
-        }
+        for (int a = 1; a < 4; ++a)
+          if ((lane & 3) == a) lrow = lam[a];
 #pragma unroll 1
         for (int c0 = 0; c0 < D; c0 += 16) {
           uint32_t r[16];
@@ -869,21 +961,16 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
       }
     }
 
-    // ---- epilogue: O / omega, lse = mu + ln(omega) ------------------------------------------------
-    if (T > 0) ok = ok && ptx::mbar_wait(&bars[kPvDone], (T - 1) & 1, status, kTimeoutCode);
+    // ---- epilogue: O / omega, lse = mu + ln(omega); each warp of the pair takes half the columns ----
+    ok = ok && ptx::mbar_wait(&bars[kFin0 + grp], 0, status, kTimeoutCode);
+    ok = ok && ptx::mbar_wait(&bars[kPvDone], (T - 1) & 1, status, kTimeoutCode);
     ptx::tc_fence_after();
-    float om_row = 1.0f, mu_row = 0.0f;
-#pragma unroll
-    for (int a = 0; a < 4; ++a) {
-      const float o = __shfl_sync(kFull, st.om[a], (lane >> 2) << 2);
-      const float m = __shfl_sync(kFull, st.mu[a], (lane >> 2) << 2);
-      if ((lane & 3) == a) { om_row = o; mu_row = m; }
-    }
-    // lane l holds row j0 + l of O: rows 4*(l>>2) + (l&3)
+    const float om_row = st_om[grp * kBQ + lane], mu_row = st_mu[grp * kBQ + lane];
     const int64_t orow = b * P.os[0] + h * P.os[1] + (int64_t)(j0 + lane) * P.os[2];
-    if (P.lse) P.lse[((int64_t)b * P.heads_q + h) * P.seqlen + j0 + lane] = (float)((double)mu_row + log((double)om_row));
+    if (side == 0 && P.lse)
+      P.lse[((int64_t)b * P.heads_q + h) * P.seqlen + j0 + lane] = (float)((double)mu_row + log((double)om_row));
 #pragma unroll 1
-    for (int c0 = 0; c0 < D; c0 += 16) {
+    for (int c0 = side * (D / 2); c0 < (side + 1) * (D / 2); c0 += 16) {
       uint32_t r[16];
       ptx::tmem_ld16(tlane + c0, r);
       ptx::tmem_wait_ld();

@@ -57,6 +57,18 @@ def test_scale_sweep_saturation(mult):
         compare_units(gpu, ref, check_stats=True, label=f"mult={mult}")
 
 
+@pytest.mark.parametrize("window,flags", [(0, 0), (192, 0), (0, oracle.FORCE_16BIT)])
+def test_head_dim_256_gemma_shaped(window, flags):
+    """head_dim 256 (two 128-channel halves per tile), global and sliding-window layers."""
+    cfg = li.CONFIGS[3]
+    q, k, v = li.make_qkv(cfg, B=1, Hq=2, Hkv=1, N=512)
+    sc = li.softmax_scale(cfg.D)
+    ref = oracle.run_all(q, k, v, scale=sc, window=window, flags=flags, dumps=True)
+    gpu = run_gpu(q, k, v, scale=sc, window=window, flags=flags, dump=(0, 1))
+    compare_units(gpu, ref, check_stats=True, label=f"D=256 window={window} flags={flags}")
+    compare_dense_bytes(gpu, ref, 0, 1)
+
+
 def test_config1_full():
     cfg = li.CONFIGS[1]
     q, k, v = li.make_qkv(cfg)
