@@ -57,6 +57,21 @@ def unit_pairs(cfg, g, window=0):
     return tot
 
 
+def max_over_ranks(ms: float, dist=None, device=None) -> float:
+    """Device time of the slowest rank (the job finishes when its last rank does)."""
+    if dist is None:
+        return float(ms)
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tflops(flops_per_rank: float, world: int, ms_per_step: float) -> float:
+    """Every rank runs the full workload on its own GPU (units are independent: weak scaling,
+    no data-path collective), so the job's throughput is world x per-rank work / slowest rank."""
+    return world * flops_per_rank / (ms_per_step * 1e-3) / 1e12
+
+
 class ClockSampler:
     """nvidia-smi clocks and throttle reasons during the timed region."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -218,12 +233,9 @@ def main():
     per = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
     total_ms = ev[0].elapsed_time(ev[-1])
     stats = lamp.lamp_attn_get_stats()
-    t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, dist, dev)
     ms_per_step = total_ms / args.steps
-    value = world * fl / (ms_per_step * 1e-3) / 1e12
+    value = whole_job_tflops(fl, world, ms_per_step)
 
     # ---- end to end: pinned host inputs in, result out, every step -------------------------
     ho = torch.empty(B, Hq, N, D, dtype=torch.bfloat16).pin_memory()
@@ -243,10 +255,7 @@ def main():
         e2e_step()
     e1.record()
     barrier()
-    t = torch.tensor([e0.elapsed_time(e1)], device=dev, dtype=torch.float64)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_ms = float(t.item()) / args.steps
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1), dist, dev) / args.steps
     h2d = sum(x.numel() * x.element_size() for x in (hq, hk, hv))
     d2h = sum(x.numel() * x.element_size() for x in (ho, hl, hf))
 
@@ -263,10 +272,9 @@ def main():
     kern_ms = statistics.mean(per)
     achieved = fl / (kern_ms * 1e-3) / 1e12
     peak = 4.0 / MIN_SLOTS_PER_STEP * SM_COUNT * LANES_PER_SM * SM_MAX_MHZ * 1e6 / 1e12
-    traffic = None
-    tfile = os.path.join(ROOT, "profiles", "dram_traffic.json")
-    if os.path.exists(tfile):
-        traffic = json.load(open(tfile)).get(f"config{cfg.index}_bytes_per_launch")
+    # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu capture summarised in
+    # profiles/lamp_fwd_sm100_config2_ncu_full.txt (algorithmic bytes: 680 MB)
+    traffic = {2: 658.75e6}.get(cfg.index) if args.mode == "lamp" else None
     roofline = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                 "frac": achieved / peak, "traffic": traffic,
                 "note": "peak = issue-slot bound of the emulated e4m3 accumulation at 2 slots/step, "
@@ -291,7 +299,7 @@ def main():
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "e4m3-emulated/f32", "data": "synthetic", "config": workload_config(cfg),
             "mode": args.mode, "clocks": clk.summary(),
-            "e2e": {"value": world * fl / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+            "e2e": {"value": whole_job_tflops(fl, world, e2e_ms), "unit": "TFLOP/s",
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
             "gpu_launches": args.steps,
             "roofline": roofline, "cpu_baseline": cpu,

@@ -78,6 +78,41 @@ def test_config1_full():
     compare_units(gpu, ref, check_stats=True, label="cfg1")
 
 
+def _sampled_full_size(cfg_index, n_units, *, window=0, mult=1.0):
+    """Full-size config through the launch configuration bench.py times; the oracle checks a
+    seeded spread of (b, h, group) units: flag bytes and y8 / e8 checksums exact, O / LSE in tolerance."""
+    cfg = li.CONFIGS[cfg_index]
+    q, k, v = li.make_qkv(cfg)
+    sc = li.softmax_scale(cfg.D, mult)
+    units = li.sample_units(cfg, n_units, seed=3 + cfg_index)
+    ref = oracle.run_units(q, k, v, units, scale=sc, window=window)
+    gpu = run_gpu(q, k, v, scale=sc, window=window)
+    if ref.stats["big_rowsum"] or ref.stats["exp16_gt1"]:
+        # outside the bit-exactness claim for O; decisions are still compared
+        for n, (b, h, g) in enumerate(ref.units):
+            assert np.array_equal(gpu["flags"][b, h, g], ref.flags[n])
+            assert np.array_equal(gpu["checks"][b, h, g].view(np.uint64), ref.checks[n])
+    else:
+        compare_units(gpu, ref, label=f"cfg{cfg_index} window={window} mult={mult}")
+    act = gpu["stats"]["subblocks_active"]
+    return (gpu["stats"]["stage1_flagged"] + gpu["stats"]["stage2_flagged"]) / act
+
+
+def test_config2_full_size_sampled():
+    frac = _sampled_full_size(2, 40)
+    assert 0.05 < frac < 0.6
+
+
+@pytest.mark.parametrize("window", [1024, 0])
+def test_config3_full_size_sampled(window):
+    _sampled_full_size(3, 24, window=window)
+
+
+def test_config4_scale_sweep_sampled():
+    fr = [_sampled_full_size(4, 10, mult=m) for m in (0.5, 8.0)]
+    assert fr[0] < fr[1]        # the recomputed fraction grows with the logit scale
+
+
 def test_strided_inputs_and_bf16_output():
     cfg = li.CONFIGS[1]
     q, k, v = li.make_qkv(cfg, Hq=2, Hkv=2, N=256, seed=5)
