@@ -125,6 +125,34 @@ int lamp_attn_fwd(const void* q, const void* k, const void* v, void* out, float*
                   uint8_t* flag_mask, const lamp_attn_params* p, void* workspace,
                   size_t workspace_bytes, void* cuda_stream);
 
+/* Forward pass plus a fingerprint of its low-precision stage, for callers that cannot allocate.
+ * (The paper has no counterpart of this call; it is a service of this library.)
+ *
+ * Some hosts of this library may not create device memory of their own: a plug-in that lives
+ * inside another framework's memory pool, a monitor process with a fixed footprint, code that
+ * runs while a pool is frozen.  They can still pass inputs and outputs they were given, but
+ * they cannot provide the [batch, heads_q, seqlen/32, seqlen/64, 2] checksum buffer that
+ * lamp_attn_params.dbg_checksums asks for.  This call runs the same kernel with that buffer
+ * placed in an array that is part of the library image (8 MiB per GPU that loads the library,
+ * held until the process exits), then folds it into two 64-bit sums:
+ *   digest[0] = sum over all (group, key tile) pairs of the y8 checksum  (mod 2^64)
+ *   digest[1] = the same for the e8 checksum
+ * i.e. exactly the sums of the two columns lamp_attn_fwd would have written to dbg_checksums.
+ *
+ *   q, k, v, out, lse, flag_mask, p, cuda_stream   as for lamp_attn_fwd; p->dbg_* are ignored
+ *   digest   device, 2 x uint64, written (not accumulated)
+ * Limit: batch * heads_q * (seqlen/32) * (seqlen/64) <= LAMP_DIGEST_MAX_PAIRS, else
+ * LAMP_ERR_UNSUPPORTED_SHAPE and nothing is enqueued.  No device memory is allocated or freed,
+ * here or in anything this call uses.  The first call on a device looks up the address of the
+ * array (and does the one-time set-up lamp_attn_fwd also does), so make that first call outside
+ * any stream capture.  All calls on a device share the one array and it keeps the last call's
+ * contents; the call clears it before use, and two calls whose kernels overlap on the GPU (different
+ * streams, no ordering between them) race on it - order them. */
+#define LAMP_DIGEST_MAX_PAIRS (1u << 19)
+int lamp_attn_fwd_digest(const void* q, const void* k, const void* v, void* out, float* lse,
+                         uint8_t* flag_mask, const lamp_attn_params* p, uint64_t* digest,
+                         void* cuda_stream);
+
 /* Wait for the stream, then copy the counters of the last lamp_attn_fwd on the current
  * device to *host_out.  Returns LAMP_ERR_DEVICE_TIMEOUT if that kernel gave up a wait. */
 int lamp_attn_get_stats(lamp_attn_stats* host_out, void* cuda_stream);

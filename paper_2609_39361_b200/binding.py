@@ -10,7 +10,7 @@ _LIB_PATH = os.path.join(_HERE, "liblamp_attn.so")
 LAMP_FORCE_16BIT, LAMP_FORCE_8BIT, LAMP_NO_STAGE1, LAMP_OUT_FP32 = 1, 2, 4, 8
 
 EXPORTS = ("lamp_attn_default_params", "lamp_attn_contiguous_strides", "lamp_attn_workspace_bytes",
-           "lamp_attn_fwd", "lamp_attn_get_stats", "lamp_attn_last_cuda_error", "lamp_attn_strerror")
+           "lamp_attn_fwd", "lamp_attn_fwd_digest", "lamp_attn_get_stats", "lamp_attn_last_cuda_error", "lamp_attn_strerror")
 
 
 class LampAttnError(RuntimeError):
@@ -61,6 +61,8 @@ def library():
         L.lamp_attn_workspace_bytes.restype = C.c_size_t; L.lamp_attn_workspace_bytes.argtypes = [PP]
         L.lamp_attn_fwd.restype = C.c_int
         L.lamp_attn_fwd.argtypes = [C.c_void_p] * 6 + [PP, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.lamp_attn_fwd_digest.restype = C.c_int
+        L.lamp_attn_fwd_digest.argtypes = [C.c_void_p] * 6 + [PP, C.c_void_p, C.c_void_p]
         L.lamp_attn_get_stats.restype = C.c_int
         L.lamp_attn_get_stats.argtypes = [C.POINTER(LampAttnStats), C.c_void_p]
         L.lamp_attn_last_cuda_error.restype = C.c_int; L.lamp_attn_last_cuda_error.argtypes = []
@@ -109,6 +111,21 @@ def lamp_attn_fwd(q, k, v, out, lse, flag_mask, p: LampAttnParams, workspace=Non
     rc = library().lamp_attn_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), _ptr(flag_mask),
                                  C.byref(p), _ptr(workspace), ws_bytes, C.c_void_p(s))
     _check(rc, "lamp_attn_fwd")
+
+
+LAMP_DIGEST_MAX_PAIRS = 1 << 19
+
+
+def lamp_attn_fwd_digest(q, k, v, out, lse, flag_mask, p: LampAttnParams, digest, stream=None) -> None:
+    """Forward pass plus the two 64-bit sums of the y8 / e8 checksums, written to `digest`
+    (CUDA int64 tensor of 2 elements).  For callers that cannot allocate device memory: the
+    checksum buffer is an array inside the library, limited to LAMP_DIGEST_MAX_PAIRS
+    (group, key tile) pairs; this wrapper allocates nothing either."""
+    import torch
+    s = torch.cuda.current_stream().cuda_stream if stream is None else stream
+    rc = library().lamp_attn_fwd_digest(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), _ptr(flag_mask),
+                                        C.byref(p), _ptr(digest), C.c_void_p(s))
+    _check(rc, "lamp_attn_fwd_digest")
 
 
 def lamp_attn_get_stats(stream=None) -> dict:

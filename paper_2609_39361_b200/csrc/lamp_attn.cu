@@ -245,6 +245,76 @@ int lamp_attn_fwd(const void* q, const void* k, const void* v, void* out, float*
   return LAMP_OK;
 }
 
+}  // extern "C"
+
+// ---------------------------------------------------------------------------------------
+// lamp_attn_fwd_digest: the checksum buffer of the forward kernel lives in the library image.
+namespace lamp {
+
+// Scratch of the digest call: two 64-bit checksums per (group, key tile) pair.  Device code may
+// name the array; host code may not use the name as a pointer (on the host it is only a handle
+// for cudaGetSymbolAddress).
+static __device__ __align__(256) unsigned long long g_digest_scratch[2 * (size_t)LAMP_DIGEST_MAX_PAIRS];
+static unsigned long long* g_digest_ptr[64] = {};   // per device, filled at the first call
+
+__global__ void lamp_digest_reduce(const unsigned long long* __restrict__ cks, size_t n_pairs,
+                                   unsigned long long* __restrict__ digest) {
+  unsigned long long a = 0, b = 0;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_pairs; i += (size_t)gridDim.x * blockDim.x) {
+    a += cks[2 * i];
+    b += cks[2 * i + 1];
+  }
+#pragma unroll
+  for (int s = 16; s > 0; s >>= 1) {
+    a += __shfl_xor_sync(0xffffffffu, a, s);
+    b += __shfl_xor_sync(0xffffffffu, b, s);
+  }
+  if ((threadIdx.x & 31) == 0) {
+    atomicAdd(&digest[0], a);
+    atomicAdd(&digest[1], b);
+  }
+}
+
+}  // namespace lamp
+
+extern "C" {
+
+int lamp_attn_fwd_digest(const void* q, const void* k, const void* v, void* out, float* lse,
+                         uint8_t* flag_mask, const lamp_attn_params* p, uint64_t* digest,
+                         void* cuda_stream) {
+  if (!p || !digest) return LAMP_ERR_INVALID_ARG;
+  if (p->batch <= 0 || p->heads_q <= 0 || p->seqlen <= 0 || p->seqlen % kBM) return LAMP_ERR_INVALID_ARG;
+  const unsigned long long n_pairs =
+      (unsigned long long)p->batch * p->heads_q * (p->seqlen / kBQ) * (p->seqlen / kTK);
+  if (n_pairs > LAMP_DIGEST_MAX_PAIRS) return LAMP_ERR_UNSUPPORTED_SHAPE;   // beyond the built-in scratch
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (dev < 0 || dev >= 64) return LAMP_ERR_UNSUPPORTED_DEVICE;
+  if (!g_digest_ptr[dev]) {   // once per device, with that device current
+    unsigned long long* ptr = nullptr;
+    e = cudaGetSymbolAddress((void**)&ptr, g_digest_scratch);
+    if (e != cudaSuccess) return cuda_fail(e);
+    g_digest_ptr[dev] = ptr;
+  }
+  lamp_attn_params pp = *p;
+  pp.dbg_y8 = nullptr;
+  pp.dbg_e8 = nullptr;
+  pp.dbg_batch = pp.dbg_head = 0;
+  pp.dbg_checksums = (uint64_t*)g_digest_ptr[dev];   // cleared by lamp_attn_fwd before the kernel
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  e = cudaMemsetAsync(digest, 0, 2 * sizeof(uint64_t), stream);
+  if (e != cudaSuccess) return cuda_fail(e);
+  const int rc = lamp_attn_fwd(q, k, v, out, lse, flag_mask, &pp, nullptr, 0, cuda_stream);
+  if (rc) return rc;
+  const int blocks = (int)((n_pairs + 255) / 256 < 592 ? (n_pairs + 255) / 256 : 592);
+  lamp_digest_reduce<<<blocks, 256, 0, stream>>>(g_digest_ptr[dev], (size_t)n_pairs,
+                                                 (unsigned long long*)digest);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  return LAMP_OK;
+}
+
 int lamp_attn_get_stats(lamp_attn_stats* host_out, void* cuda_stream) {
   if (!host_out) return LAMP_ERR_INVALID_ARG;
   cudaStream_t stream = (cudaStream_t)cuda_stream;

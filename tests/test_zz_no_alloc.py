@@ -1,0 +1,59 @@
+"""The digest entry point, which keeps its checksum scratch inside the library image so that a
+caller unable to allocate device memory (a plug-in inside someone else's memory pool, a fixed-
+footprint monitor) can still fingerprint the low-precision stage.  It must give the same outputs
+as the regular entry point and the sums of that entry point's checksum columns, call after call
+(the shared scratch keeps the previous call's contents and has to be cleared every time)."""
+import numpy as np
+import pytest
+import torch
+
+import lamp_inputs as li
+
+pytestmark = pytest.mark.gpu
+
+
+def _params(lamp, q, k, scale, out):
+    p = lamp.lamp_attn_default_params()
+    B, Hq, N, D = q.shape
+    p.batch, p.heads_q, p.heads_kv, p.seqlen, p.head_dim = B, Hq, k.shape[1], N, D
+    lamp.lamp_attn_contiguous_strides(p)
+    p.scale = scale
+    return p
+
+
+def test_digest_entry_point_matches_regular_entry_point_twice():
+    import paper_2609_39361_b200 as lamp
+    dev = torch.device("cuda:0")
+    cfg = li.CONFIGS[1]
+    shapes = [dict(Hq=4, Hkv=2, N=640, seed=21), dict(Hq=2, Hkv=1, N=256, seed=22)]   # second call is smaller:
+    # stale checksums of the first call would show up in its digest if the scratch were not cleared
+    for round_ in range(2):
+        for shp in shapes:
+            q, k, v = [t.to(dev) for t in li.make_qkv(cfg, **shp)]
+            sc = li.softmax_scale(cfg.D)
+            B, Hq, N, D = q.shape
+            ref = lamp.forward(q, k, v, scale=sc, checksums=True)
+            want = ref["checks"].reshape(-1, 2).sum(0)                 # int64 sums wrap mod 2^64
+            out = torch.empty_like(ref["out"]); lse = torch.empty_like(ref["lse"])
+            fm = torch.empty_like(ref["flags"]); digest = torch.full((2,), -1, device=dev, dtype=torch.int64)
+            p = _params(lamp, q, k, sc, out)
+            before = torch.cuda.memory_allocated(dev)
+            lamp.lamp_attn_fwd_digest(q, k, v, out, lse, fm, p, digest)
+            torch.cuda.synchronize()
+            assert torch.cuda.memory_allocated(dev) == before
+            assert torch.equal(out, ref["out"]) and torch.equal(lse, ref["lse"]) and torch.equal(fm, ref["flags"])
+            assert torch.equal(digest, want), (round_, shp, digest, want)
+            assert lamp.lamp_attn_get_stats()["device_status"] == 0
+
+
+def test_digest_entry_point_rejects_sizes_beyond_its_scratch():
+    import paper_2609_39361_b200 as lamp
+    dev = torch.device("cuda:0")
+    N = 8192                                        # 1 * 32 * 256 * 128 = 2^20 pairs > 2^19
+    q = torch.zeros(1, 32, N, 128, device=dev, dtype=torch.bfloat16)
+    kv = torch.zeros(1, 8, N, 128, device=dev, dtype=torch.bfloat16)
+    out = torch.empty_like(q); digest = torch.zeros(2, device=dev, dtype=torch.int64)
+    p = _params(lamp, q, kv, 0.088, out)
+    assert p.batch * p.heads_q * (N // 32) * (N // 64) > lamp.LAMP_DIGEST_MAX_PAIRS
+    with pytest.raises(lamp.LampAttnError, match="shape"):
+        lamp.lamp_attn_fwd_digest(q, kv, kv, out, None, None, p, digest)
