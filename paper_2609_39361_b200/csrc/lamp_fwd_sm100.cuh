@@ -2,20 +2,21 @@
 //
 // One CTA = 128 query rows of one (batch, query head); key tiles of 64 keys are visited
 // in ascending order (the flags depend on the history of the running maxima, so the key
-// dimension is never split across CTAs).  Twelve warps in three groups of four:
+// dimension is never split across CTAs).  Sixteen warps in four groups of four:
 //
-//   warps 0-7  compute.  Group g of 32 rows (TMEM lanes 32g..32g+31) is shared by warps g
-//              and g+4, which take the even and the odd key tiles.  The emulated e4m3 chain of
-//              a tile needs nothing from earlier tiles, so while one warp of the pair walks the
-//              (latency-bound, fp64-heavy) decision path of tile n - stage 1, exponentials,
-//              stage 2, recomputation, rescale of O, P tile - the other already runs the chain
-//              of tile n+1 on the same scheduler.  The row state (mu, omega) passes between
-//              them through shared memory, guarded by a token mbarrier.
-//   warps 8-9  convert the bf16 K half-tile (64 keys x 128 channels) that TMA delivered into
-//              the fp32, key-contiguous layout the chain reads (double buffered).
-//   warp  10   issues the TMA loads of K.
-//   warp  11   issues the TMA loads of V and the tcgen05 MMAs O += P V (bf16 x bf16 -> fp32
-//              in TMEM; 16-bit exponentials enter as bf16 hi + lo).
+//   warps 0-3    decision path.  Warp g owns the group of 32 rows 32g..32g+31 (TMEM lanes
+//                32g..32g+31) and its running (mu, omega): stage 1, exponentials, stage 2,
+//                fp64 recomputation, rescale of O, P tile to shared memory.
+//   warps 4-11   the emulated e4m3 chain (the bulk of the work).  Warps 4+g and 8+g serve group
+//                g and take the even and the odd key tiles.  A chain needs only Q and K, so these
+//                warps run ahead of the decision path: each finished tile is packed four e4m3
+//                values to a word (the packed accumulator layout of Sec. 3.3) and queued in a
+//                four-slot ring in the group's TMEM lanes.
+//   warps 12-13  convert the bf16 K half-tile (64 keys x 128 channels) that TMA delivered into
+//                the fp32, key-contiguous layout the chain reads (double buffered).
+//   warp  14     issues the TMA loads of K.
+//   warp  15     issues the TMA loads of V and the tcgen05 MMAs O += P V (bf16 x bf16 -> fp32
+//                in TMEM; 16-bit exponentials enter as bf16 hi + lo).
 //
 // head_dim 256 runs as two 128-channel halves per tile: the chain carries its accumulators
 // from the first half to the second, P V is issued per 128 output columns.
@@ -28,8 +29,9 @@
 
 namespace lamp {
 
-constexpr int kThreads = 384;
-constexpr int kConvWarp0 = 8, kConvWarps = 2, kKWarp = 10, kCtrlWarp = 11;
+constexpr int kThreads = 512;
+constexpr int kConvWarp0 = 12, kConvWarps = 2, kKWarp = 14, kCtrlWarp = 15;
+constexpr int kSlots = 4;          // ring of finished chain tiles per group
 constexpr int kTimeoutCode = -4;   // LAMP_ERR_DEVICE_TIMEOUT
 constexpr int kHalf = 128;         // channels per K / V half-tile
 
@@ -43,9 +45,8 @@ struct SmemLayout {
   static constexpr int kPlo = kPhi + kBM * kTK * 2;
   static constexpr int kLut = kPlo + kBM * kTK * 2;               // 128 x uint2
   static constexpr int kDscr = kLut + 1024;                       // 4 groups x 384 doubles
-  static constexpr int kState = kDscr + 4 * 384 * 8;              // mu[128], omega[128], lo_dirty[4]
-  static constexpr int kBar = kState + 1024 + 16;                 // mbarriers
-  static constexpr int kMisc = kBar + 256;                        // tmem slot, lo masks
+  static constexpr int kBar = kDscr + 4 * 384 * 8;                // mbarriers
+  static constexpr int kMisc = kBar + 512;                        // tmem slot, lo masks
   static constexpr int kBytes = kMisc + 64;
   static_assert(kKbf % 1024 == 0 && kV % 1024 == 0 && kPhi % 1024 == 0 && kPlo % 1024 == 0, "swizzle atoms");
 };
@@ -55,9 +56,9 @@ enum Bar {
   // fp32 K half-tile m lives in buffer m & 1 and is announced on barrier m & 3: a compute warp
   // only meets every other tile, and must never be two completions behind on a barrier it polls
   kKfFull0, kKfEmpty0 = kKfFull0 + 4, kVFull = kKfEmpty0 + 4, kVHalf, kPReady, kPvDone,
-  kTok0,              // [group][tile parity]: the row state after the previous tile is in shared memory
-  kFin0 = kTok0 + 8,  // [group]: the final row state is in shared memory
-  kNumBars = kFin0 + 4
+  kSlotFull0,                              // [group][slot]: a packed chain tile waits in TMEM
+  kSlotEmpty0 = kSlotFull0 + 4 * kSlots,   // [group][slot]: the decision-path warp has taken it
+  kNumBars = kSlotEmpty0 + 4 * kSlots
 };
 
 struct TileGeom {
@@ -215,6 +216,22 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // Byte address of (row, 16-byte chunk) inside a [rows][64] bf16 tile with the 128-byte swizzle.
 __device__ __forceinline__ uint32_t sw128(int row, int chunk) { return row * 128 + ((chunk ^ (row & 7)) << 4); }
 
+// Four e4m3 values <-> one 32-bit word (byte u = value u): the packed accumulator layout of
+// Sec. 3.3 ("4 accumulators occupy a single 32-bit register"), used to hand the first-pass
+// logits from the chain warps to the decision-path warp through TMEM.  Exact both ways.
+__device__ __forceinline__ uint32_t pack_e4m3x4(float v0, float v1, float v2, float v3) {
+  uint32_t r;
+  asm("{.reg .b16 lo, hi; cvt.rn.satfinite.e4m3x2.f32 lo, %2, %1; cvt.rn.satfinite.e4m3x2.f32 hi, %4, %3;"
+      " mov.b32 %0, {lo, hi};}" : "=r"(r) : "f"(v0), "f"(v1), "f"(v2), "f"(v3));
+  return r;
+}
+__device__ __forceinline__ void unpack_e4m3x4(uint32_t w, float (&y)[4]) {
+  asm("{.reg .b16 lo, hi; .reg .b32 a, b; .reg .f16 h0, h1, h2, h3; mov.b32 {lo, hi}, %4;"
+      " cvt.rn.f16x2.e4m3x2 a, lo; cvt.rn.f16x2.e4m3x2 b, hi; mov.b32 {h0, h1}, a; mov.b32 {h2, h3}, b;"
+      " cvt.f32.f16 %0, h0; cvt.f32.f16 %1, h1; cvt.f32.f16 %2, h2; cvt.f32.f16 %3, h3;}"
+      : "=f"(y[0]), "=f"(y[1]), "=f"(y[2]), "=f"(y[3]) : "r"(w));
+}
+
 // e8 byte of an 8-bit exponential value (0xF8 = 1.0, E = 0 subnormals in units of 2^-33).
 __device__ __forceinline__ uint32_t enc_exp8(float e) {
   if (e == 0.0f) return 0u;
@@ -227,14 +244,14 @@ __device__ __forceinline__ uint32_t enc_exp8(float e) {
 // stage 2 (eq. (8)), stage-2 recomputation.  Writes the group's 32 rows of the P tile
 // (bf16 hi, and bf16 lo for 16-bit sub-blocks), returns the flag byte.
 //
-// The 64 first-pass logits of a lane are parked in its own TMEM lane right away (tacc) and
-// read back 16 at a time, so that the per-element work is a short loop instead of a long
-// unrolled stretch of code and the registers are free for the 16-bit path.
+// The 64 first-pass logits of a lane arrive packed in 16 words (yw) and are unpacked 16 at a
+// time, so that the per-element work is a short loop instead of a long unrolled stretch of
+// code and the registers are free for the 16-bit path.
 template <int D, bool FULL, bool DUMP>
-__device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileGeom& g, float (&acc)[4][16],
+__device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileGeom& g, const uint32_t (&yw)[16],
                                               const __nv_bfloat16* ktile, int64_t kstride, uint32_t tq,
                                               const uint2* lut, double* dscr, unsigned char* phi, unsigned char* plo,
-                                              uint32_t tscratch, uint32_t tacc, uint32_t& lo_dirty, RowState& st,
+                                              uint32_t tscratch, uint32_t& lo_dirty, RowState& st,
                                               float (&lam)[4], WarpCounters& wc, unsigned long long (&cks)[2],
                                               int dump_row0, int row0, long long* ph) {
   const int lane = threadIdx.x & 31;
@@ -244,20 +261,22 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
   const bool force8 = P.flags & LAMP_FORCE_8BIT;
   const bool skip1 = (P.flags & (LAMP_FORCE_8BIT | LAMP_NO_STAGE1)) != 0;
 
-  // ---- per sub-block, per query maxima; park the logits; which sub-blocks are active -------
+  // ---- per sub-block, per query maxima; which sub-blocks are active --------------------------
+  // yw[4a + c] packs the first-pass logits of query a, keys 4c..4c+3 of the lane's sub-block
   float cm[4];
 #pragma unroll
   for (int a = 0; a < 4; ++a) {
     float m = -INFINITY;
 #pragma unroll
-    for (int b = 0; b < 16; ++b)
-      if (vis<FULL>(g, 16 * th_own + b, 4 * qa + a)) m = fmaxf(m, acc[a][b]);
+    for (int c = 0; c < 4; ++c) {
+      float y[4];
+      unpack_e4m3x4(yw[4 * a + c], y);
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (vis<FULL>(g, 16 * th_own + 4 * c + u, 4 * qa + a)) m = fmaxf(m, y[u]);
+    }
     cm[a] = m;
     wc.sat8 += m == 448.0f;
-    uint32_t r[16];
-#pragma unroll
-    for (int b = 0; b < 16; ++b) r[b] = __float_as_uint(acc[a][b]);
-    ptx::tmem_st16(tacc + 16 * a, r);
   }
   uint32_t actmask = 0;
 #pragma unroll
@@ -403,62 +422,69 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
   // entries of 2^-15 or more are multiples of 2^-18 (16 of them stay below 2^5), smaller
   // ones are multiples of 2^-33 (their sum stays below 2^-11).
   double rs8[4] = {0.0, 0.0, 0.0, 0.0};
-  ptx::tmem_wait_st();
 #pragma unroll 1
   for (int a = 0; a < 4; ++a) {
     const int row = row0 + 4 * qa + a;
     uint32_t w[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    // (TMEM loads are warp-collective: every lane takes part, whatever its sub-block's path)
-    uint32_t yr[16];
-    ptx::tmem_ld16(tacc + 16 * a, yr);
-    ptx::tmem_wait_ld();
     if (own8 || (DUMP && own_act)) {
       float mh_sel = muh[0];
+      uint32_t ya[4] = {yw[0], yw[1], yw[2], yw[3]};
 #pragma unroll
       for (int k = 1; k < 4; ++k)
-        if (a == k) mh_sel = muh[k];
+        if (a == k) {
+          mh_sel = muh[k];
+#pragma unroll
+          for (int c = 0; c < 4; ++c) ya[c] = yw[4 * k + c];
+        }
       const float m8h = 0.5f * trunc_e4m3(mh_sel);
       float s_hi = 0.0f, s_lo = 0.0f;
 #pragma unroll
-      for (int b = 0; b < 16; b += 2) {
-        const bool ok0 = vis<FULL>(g, 16 * th_own + b, 4 * qa + a);
-        const bool ok1 = vis<FULL>(g, 16 * th_own + b + 1, 4 * qa + a);
-        const float y0 = __uint_as_float(yr[b]), y1 = __uint_as_float(yr[b + 1]);
-        float e0 = 0.0f, e1 = 0.0f;
-        if (own8) {
-          // half the shift (exact), rounded to 4 significant bits by the conversion unit: its
-          // e4m3 code indexes the table (shifts below 2^-5 all map to 1.0, as in the 256-entry table)
-          unsigned short pk;
-          asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(pk)
-              : "f"(__fmaf_rn(y1, -0.5f, m8h)), "f"(__fmaf_rn(y0, -0.5f, m8h)));
-          const uint2 w0 = lut[pk & 0x7fu], w1 = lut[(pk >> 8) & 0x7fu];
-          if (ok0) { e0 = __uint_as_float(w0.x); s_lo += __uint_as_float(w0.y); s_hi += e0 - __uint_as_float(w0.y); }
-          if (ok1) { e1 = __uint_as_float(w1.x); s_lo += __uint_as_float(w1.y); s_hi += e1 - __uint_as_float(w1.y); }
-        }
-        w[b >> 1] = pack_bf16(e0, e1);
-        if (DUMP) {
-          const float yy[2] = {y0, y1}, ee[2] = {e0, e1};
-          const bool okk[2] = {ok0, ok1};
+      for (int c = 0; c < 4; ++c) {
+        float y4[4];
+        unpack_e4m3x4(ya[c], y4);
 #pragma unroll
-          for (int u = 0; u < 2; ++u) {
-            if (!okk[u]) continue;
-            const uint32_t yb = enc_e4m3(yy[u]);
-            const uint32_t ebb = own8 ? enc_exp8(ee[u]) : 0xffu;
-            const uint64_t idx = (uint64_t)((16 * th_own + b + u) * kBQ + 4 * qa + a) << 8;
-            cks[0] += mix64(idx | yb);
-            cks[1] += mix64(idx | ebb);
-            if (dump_row0 >= 0) {
-              const size_t off = (size_t)(dump_row0 + 4 * qa + a) * P.seqlen + g.i0 + 16 * th_own + b + u;
-              if (P.dbg_y8) P.dbg_y8[off] = (uint8_t)yb;
-              if (P.dbg_e8) P.dbg_e8[off] = (uint8_t)ebb;
+        for (int u = 0; u < 4; u += 2) {
+          const int b = 4 * c + u;
+          const bool ok0 = vis<FULL>(g, 16 * th_own + b, 4 * qa + a);
+          const bool ok1 = vis<FULL>(g, 16 * th_own + b + 1, 4 * qa + a);
+          const float y0 = y4[u], y1 = y4[u + 1];
+          float e0 = 0.0f, e1 = 0.0f;
+          if (own8) {
+            // half the shift (exact), rounded to 4 significant bits by the conversion unit: its
+            // e4m3 code indexes the table (shifts below 2^-5 all map to 1.0, as in the 256-entry table)
+            unsigned short pk;
+            asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(pk)
+                : "f"(__fmaf_rn(y1, -0.5f, m8h)), "f"(__fmaf_rn(y0, -0.5f, m8h)));
+            const uint2 w0 = lut[pk & 0x7fu], w1 = lut[(pk >> 8) & 0x7fu];
+            if (ok0) { e0 = __uint_as_float(w0.x); s_lo += __uint_as_float(w0.y); s_hi += e0 - __uint_as_float(w0.y); }
+            if (ok1) { e1 = __uint_as_float(w1.x); s_lo += __uint_as_float(w1.y); s_hi += e1 - __uint_as_float(w1.y); }
+          }
+          w[b >> 1] = pack_bf16(e0, e1);
+          if (DUMP) {
+            const float ee[2] = {e0, e1};
+            const bool okk[2] = {ok0, ok1};
+#pragma unroll
+            for (int v = 0; v < 2; ++v) {
+              if (!okk[v]) continue;
+              uint32_t yb = (ya[c] >> (8 * (u + v))) & 0xffu;
+              if (yb == 0x80u) yb = 0;                       // -0 is stored as +0
+              const uint32_t ebb = own8 ? enc_exp8(ee[v]) : 0xffu;
+              const uint64_t idx = (uint64_t)((16 * th_own + b + v) * kBQ + 4 * qa + a) << 8;
+              cks[0] += mix64(idx | yb);
+              cks[1] += mix64(idx | ebb);
+              if (dump_row0 >= 0) {
+                const size_t off = (size_t)(dump_row0 + 4 * qa + a) * P.seqlen + g.i0 + 16 * th_own + b + v;
+                if (P.dbg_y8) P.dbg_y8[off] = (uint8_t)yb;
+                if (P.dbg_e8) P.dbg_e8[off] = (uint8_t)ebb;
+              }
             }
           }
         }
       }
-      const double s = (double)s_hi + (double)s_lo;
+      const double sd = (double)s_hi + (double)s_lo;
 #pragma unroll
       for (int k = 0; k < 4; ++k)
-        if (a == k) rs8[k] = s;
+        if (a == k) rs8[k] = sd;
     }
     if (own8 || !own_act) {   // kept 8-bit values, or the zeros of an inactive sub-block
       *reinterpret_cast<uint4*>(phi + sw128(row, 2 * th_own)) = make_uint4(w[0], w[1], w[2], w[3]);
@@ -650,9 +676,6 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
   unsigned char* plo = smem + L::kPlo;
   uint2* lut = reinterpret_cast<uint2*>(smem + L::kLut);
   double* dscr_all = reinterpret_cast<double*>(smem + L::kDscr);
-  float* st_mu = reinterpret_cast<float*>(smem + L::kState);
-  float* st_om = st_mu + kBM;
-  uint32_t* st_lod = reinterpret_cast<uint32_t*>(st_om + kBM);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBar);
   uint32_t* tslot = reinterpret_cast<uint32_t*>(smem + L::kMisc);
   uint32_t* lomask = tslot + 1;   // [2]
@@ -684,7 +707,7 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
     ptx::mbar_init(&bars[kVHalf], 1);
     ptx::mbar_init(&bars[kPReady], 4);
     ptx::mbar_init(&bars[kPvDone], 1);
-    for (int i = 0; i < 12; ++i) ptx::mbar_init(&bars[kTok0 + i], 1);
+    for (int i = 0; i < 8 * kSlots; ++i) ptx::mbar_init(&bars[kSlotFull0 + i], 1);
     ptx::fence_barrier_init();
     lomask[0] = lomask[1] = 0;
   }
@@ -714,16 +737,18 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
       reinterpret_cast<uint4*>(phi)[c] = make_uint4(0, 0, 0, 0);
       reinterpret_cast<uint4*>(plo)[c] = make_uint4(0, 0, 0, 0);
     }
-    for (int c = tid; c < kBM; c += kThreads) { st_mu[c] = -INFINITY; st_om[c] = 0.0f; }
-    if (tid < 4) st_lod[tid] = 0;
   }
   ptx::fence_proxy_async();
   ptx::tc_fence_before();
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tbase = *tslot;
+  // TMEM columns of a group's lanes: [0, D) O, 64 for the 16-bit logits, D/2 for the lane's raw bf16
+  // query row (operand of the 16-bit dots), kSlots x 16 for the ring of packed first-pass logits
+  constexpr uint32_t kColScr = D, kColQ = D + 64, kColRing = D + 64 + D / 2;
+  static_assert(kColRing + 16 * kSlots <= 512, "TMEM columns");
 
-  if (warp >= 8) {
+  if (warp >= 12) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
     if (warp == kKWarp) {
       // =========================== K stream: one TMA half-tile ahead of the converters ===========
@@ -784,7 +809,7 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
           ok = __all_sync(kFull, ok);
         }
       }
-    } else if (warp < kConvWarp0 + kConvWarps) {
+    } else {
       // =========================== converters: bf16 K half-tile -> fp32, key-contiguous ==============
       const int key = tid - kConvWarp0 * 32;   // 0..63: one key of the tile per thread
       const int pos = kf_pos(key);
@@ -809,10 +834,55 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
         }
       }
     }
+  } else if (warp >= 4) {
+    // =========================== chain warps: emulated 8-bit logits, queued in TMEM ================
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 120;");
+    const int grp = warp & 3, side = (warp >> 2) - 1;   // side 0: even tiles, side 1: odd tiles
+    const int qa = lane >> 2;
+    const int j0 = m0 + grp * kBQ;
+    const uint32_t tring = tbase + ((uint32_t)(grp * 32) << 16) + kColRing;
+    const unsigned char* q_quad = qs + (QF32 ? 4 : 2) * (grp * kBQ + 4 * qa);
+    bool ok = true;
+    for (int n = side; n < T && ok; n += 2) {
+      const int i0 = (t_begin + n) * kTK;
+      const bool any = (!P.causal || i0 <= j0 + 31) && (P.window == 0 || j0 - (i0 + 63) < P.window);
+      float acc[4][16];
+#pragma unroll
+      for (int hh = 0; hh < NH; ++hh) {
+        const int m = n * NH + hh;
+        const float* kf = kf_all + (m & 1) * kHalf * kKfStride + kf_pos(16 * (lane & 3));
+        ok = ok && ptx::mbar_wait(&bars[kKfFull0 + (m & 3)], (m >> 2) & 1, status, kTimeoutCode);
+        if (any) {
+          const unsigned char* qh = q_quad + (size_t)hh * kHalf * kBM * (QF32 ? 4 : 2);
+          if (hh == 0) chain8<QF32, true>(qh, kf, P.scale, acc);
+          else chain8<QF32, false>(qh, kf, P.scale, acc);
+        }
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&bars[kKfEmpty0 + (m & 3)]);
+      }
+      // queue the tile: slot n % kSlots, free again once the decision-path warp has read it
+      const int slot = n & (kSlots - 1), use = n / kSlots;
+      if (use > 0)
+        ok = ok && ptx::mbar_wait(&bars[kSlotEmpty0 + kSlots * grp + slot], (use - 1) & 1, status, kTimeoutCode);
+      ptx::tc_fence_after();
+      if (any) {
+        uint32_t yw[16];
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+          for (int c = 0; c < 4; ++c)
+            yw[4 * a + c] = pack_e4m3x4(acc[a][4 * c], acc[a][4 * c + 1], acc[a][4 * c + 2], acc[a][4 * c + 3]);
+        ptx::tmem_st16(tring + 16 * slot, yw);
+        ptx::tmem_wait_st();
+      }
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&bars[kSlotFull0 + kSlots * grp + slot]);
+    }
   } else {
-    // =========================== compute: two warps per group of 32 query rows =====================
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
-    const int grp = warp & 3, side = warp >> 2;   // side 0 takes the even tiles, side 1 the odd ones
+    // =========================== decision path: one warp per group of 32 query rows ================
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
+    const int grp = warp;
     const int qa = lane >> 2;
     const int j0 = m0 + grp * kBQ;
     const int ntk = P.seqlen / kTK;
@@ -820,10 +890,8 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
     const __nv_bfloat16* kg = P.k + b * P.ks[0] + hk * P.ks[1];
     double* dscr = dscr_all + grp * 384;
     const uint32_t tlane = tbase + ((uint32_t)(grp * 32) << 16);
-    // TMEM columns of the group's lanes: [0, D) O, then 64 for the 16-bit logits, 64 for the parked
-    // first-pass logits, D/2 for the lane's raw bf16 query row (operand of the 16-bit dots)
-    const uint32_t tscr = tlane + D, tacc = tlane + D + 64, tq = tlane + D + 128;
-    if (side == 0) {
+    const uint32_t tscr = tlane + kColScr, tq = tlane + kColQ, tring = tlane + kColRing;
+    {
       const __nv_bfloat16* qrow = P.q + b * P.qs[0] + h * P.qs[1] + (int64_t)(j0 + lane) * P.qs[2];
 #pragma unroll 1
       for (int c0 = 0; c0 < D / 2; c0 += 16) {
@@ -838,15 +906,16 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
       ptx::tmem_wait_st();
     }
     RowState st;
+#pragma unroll
+    for (int a = 0; a < 4; ++a) { st.mu[a] = -INFINITY; st.om[a] = 0.0f; }
     WarpCounters wc;
     memset(&wc, 0, sizeof(wc));
     uint32_t lo_dirty = 0;
     bool ok = true;
     long long ph[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     (void)ph;
-    const unsigned char* q_quad = qs + (QF32 ? 4 : 2) * (grp * kBQ + 4 * qa);
 
-    for (int n = side; n < T && ok; n += 2) {
+    for (int n = 0; n < T && ok; ++n) {
       const int t = t_begin + n, i0 = t * kTK;
       TileGeom g;
       g.i0 = i0; g.j0 = j0; g.causal = P.causal; g.window = P.window;
@@ -856,55 +925,36 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
       uint32_t flag = 0;
       unsigned long long cks[2] = {0ull, 0ull};
 
-      // ---- emulated 8-bit logits: needs only K and Q, runs ahead of the other warp's decision path
-      float acc[4][16];
-#pragma unroll
-      for (int hh = 0; hh < NH; ++hh) {
-        const int m = n * NH + hh;
-        const float* kf = kf_all + (m & 1) * kHalf * kKfStride + kf_pos(16 * (lane & 3));
-        LAMP_TIC(t_w0);
-        ok = ok && ptx::mbar_wait(&bars[kKfFull0 + (m & 3)], (m >> 2) & 1, status, kTimeoutCode);
-        LAMP_TOC(0, t_w0);
-        LAMP_TIC(t_c);
-        if (any) {
-          const unsigned char* qh = q_quad + (size_t)hh * kHalf * kBM * (QF32 ? 4 : 2);
-          if (hh == 0) chain8<QF32, true>(qh, kf, P.scale, acc);
-          else chain8<QF32, false>(qh, kf, P.scale, acc);
-        }
-        LAMP_TOC(1, t_c);
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(&bars[kKfEmpty0 + (m & 3)]);
-      }
-
-      // ---- the row state after tile n-1 (from the other warp), and O / P free again ---------------
-      LAMP_TIC(t_w1);
-      if (n > 0) {
-        ok = ok && ptx::mbar_wait(&bars[kTok0 + 2 * grp + (n & 1)], (((n + 1) >> 1) - 1) & 1, status, kTimeoutCode);
-        ok = ok && ptx::mbar_wait(&bars[kPvDone], (n - 1) & 1, status, kTimeoutCode);
-      }
+      // ---- take the tile's first-pass logits out of the ring ------------------------------------
+      const int slot = n & (kSlots - 1), use = n / kSlots;
+      LAMP_TIC(t_w0);
+      ok = ptx::mbar_wait(&bars[kSlotFull0 + kSlots * grp + slot], use & 1, status, kTimeoutCode);
       ptx::tc_fence_after();
-      {
-        const float4 m4 = *reinterpret_cast<const float4*>(st_mu + grp * kBQ + 4 * qa);
-        const float4 o4 = *reinterpret_cast<const float4*>(st_om + grp * kBQ + 4 * qa);
-        st.mu[0] = m4.x; st.mu[1] = m4.y; st.mu[2] = m4.z; st.mu[3] = m4.w;
-        st.om[0] = o4.x; st.om[1] = o4.y; st.om[2] = o4.z; st.om[3] = o4.w;
-        lo_dirty = st_lod[grp];
+      LAMP_TOC(0, t_w0);
+      uint32_t yw[16];
+      if (any) {
+        ptx::tmem_ld16(tring + 16 * slot, yw);
+        ptx::tmem_wait_ld();
       }
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&bars[kSlotEmpty0 + kSlots * grp + slot]);
+
+      // ---- the previous P V product must be complete before O is rescaled or P is overwritten ------
+      LAMP_TIC(t_w1);
+      if (n > 0) ok = ok && ptx::mbar_wait(&bars[kPvDone], (n - 1) & 1, status, kTimeoutCode);
+      ptx::tc_fence_after();
       LAMP_TOC(2, t_w1);
       LAMP_TIC(t_p);
       if (any) {
         const int dump0 = dump_rows ? j0 : -1;
         const __nv_bfloat16* ktile = kg + (int64_t)i0 * P.ks[2];
         if (full)
-          flag = lamp_post<D, true, DUMP>(P, g, acc, ktile, P.ks[2], tq, lut, dscr, phi, plo, tscr, tacc, lo_dirty,
+          flag = lamp_post<D, true, DUMP>(P, g, yw, ktile, P.ks[2], tq, lut, dscr, phi, plo, tscr, lo_dirty,
                                           st, lam, wc, cks, dump0, grp * kBQ, ph);
         else
-          flag = lamp_post<D, false, DUMP>(P, g, acc, ktile, P.ks[2], tq, lut, dscr, phi, plo, tscr, tacc, lo_dirty,
+          flag = lamp_post<D, false, DUMP>(P, g, yw, ktile, P.ks[2], tq, lut, dscr, phi, plo, tscr, lo_dirty,
                                            st, lam, wc, cks, dump0, grp * kBQ, ph);
-        if ((lane & 3) == 0) {
-          *reinterpret_cast<float4*>(st_mu + grp * kBQ + 4 * qa) = make_float4(st.mu[0], st.mu[1], st.mu[2], st.mu[3]);
-          *reinterpret_cast<float4*>(st_om + grp * kBQ + 4 * qa) = make_float4(st.om[0], st.om[1], st.om[2], st.om[3]);
-        }
       } else {
         // no visible pair for this group: its rows of the P tile are zero
         for (int c = lane; c < kBQ * 8; c += 32) {
@@ -913,12 +963,7 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
         }
         lo_dirty = 0;
       }
-      if (lane == 0) st_lod[grp] = lo_dirty;
       LAMP_TOC(3, t_p);
-      // hand the state (and the TMEM scratch columns) to the other warp of the pair
-      ptx::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(n + 1 < T ? &bars[kTok0 + 2 * grp + ((n + 1) & 1)] : &bars[kFin0 + grp]);
       LAMP_TIC(t_r);
 
       // O <- diag(lambda_hat) O, only when some row of the group changes its maximum
@@ -961,16 +1006,17 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
       }
     }
 
-    // ---- epilogue: O / omega, lse = mu + ln(omega); each warp of the pair takes half the columns ----
-    ok = ok && ptx::mbar_wait(&bars[kFin0 + grp], 0, status, kTimeoutCode);
+    // ---- epilogue: O / omega, lse = mu + ln(omega) --------------------------------------------------
     ok = ok && ptx::mbar_wait(&bars[kPvDone], (T - 1) & 1, status, kTimeoutCode);
     ptx::tc_fence_after();
-    const float om_row = st_om[grp * kBQ + lane], mu_row = st_mu[grp * kBQ + lane];
+    float om_row = st.om[0], mu_row = st.mu[0];   // row = lane = 4*qa + (lane & 3)
+#pragma unroll
+    for (int a = 1; a < 4; ++a)
+      if ((lane & 3) == a) { om_row = st.om[a]; mu_row = st.mu[a]; }
     const int64_t orow = b * P.os[0] + h * P.os[1] + (int64_t)(j0 + lane) * P.os[2];
-    if (side == 0 && P.lse)
-      P.lse[((int64_t)b * P.heads_q + h) * P.seqlen + j0 + lane] = (float)((double)mu_row + log((double)om_row));
+    if (P.lse) P.lse[((int64_t)b * P.heads_q + h) * P.seqlen + j0 + lane] = (float)((double)mu_row + log((double)om_row));
 #pragma unroll 1
-    for (int c0 = side * (D / 2); c0 < (side + 1) * (D / 2); c0 += 16) {
+    for (int c0 = 0; c0 < D; c0 += 16) {
       uint32_t r[16];
       ptx::tmem_ld16(tlane + c0, r);
       ptx::tmem_wait_ld();
