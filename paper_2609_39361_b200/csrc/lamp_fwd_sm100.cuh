@@ -253,7 +253,8 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
                                               const uint2* lut, double* dscr, unsigned char* phi, unsigned char* plo,
                                               uint32_t tscratch, uint32_t& lo_dirty, RowState& st,
                                               float (&lam)[4], WarpCounters& wc, unsigned long long (&cks)[2],
-                                              int dump_row0, int row0, long long* ph) {
+                                              int dump_row0, int row0, long long* ph, uint64_t* pv_bar,
+                                              uint32_t pv_parity, bool pv_wait, int* status, bool& ok) {
   const int lane = threadIdx.x & 31;
   const int qa = lane >> 2, th_own = lane & 3;
   const double scale_d = (double)P.scale;
@@ -366,6 +367,16 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
       m = fmaxf(m, __shfl_xor_sync(kFull, m, 2));
       muh[a] = fmaxf(muh[a], m);
     }
+  }
+
+  // Everything up to here touched neither O nor the P tile.  From here on P is rewritten, so the
+  // previous tile's P V product (all four groups) must have completed; waiting only now lets this
+  // group's 16-bit logits overlap with the other groups' tails.
+  {
+    LAMP_TIC(t_w1);
+    if (pv_wait) ok = ok && ptx::mbar_wait(pv_bar, pv_parity, status, kTimeoutCode);
+    ptx::tc_fence_after();
+    LAMP_TOC(2, t_w1);
   }
 
   // ---- exponentials ---------------------------------------------------------------------------
@@ -940,23 +951,23 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&bars[kSlotEmpty0 + kSlots * grp + slot]);
 
-      // ---- the previous P V product must be complete before O is rescaled or P is overwritten ------
-      LAMP_TIC(t_w1);
-      if (n > 0) ok = ok && ptx::mbar_wait(&bars[kPvDone], (n - 1) & 1, status, kTimeoutCode);
-      ptx::tc_fence_after();
-      LAMP_TOC(2, t_w1);
       LAMP_TIC(t_p);
       if (any) {
         const int dump0 = dump_rows ? j0 : -1;
         const __nv_bfloat16* ktile = kg + (int64_t)i0 * P.ks[2];
         if (full)
           flag = lamp_post<D, true, DUMP>(P, g, yw, ktile, P.ks[2], tq, lut, dscr, phi, plo, tscr, lo_dirty,
-                                          st, lam, wc, cks, dump0, grp * kBQ, ph);
+                                          st, lam, wc, cks, dump0, grp * kBQ, ph, &bars[kPvDone], (n - 1) & 1, n > 0,
+                                          status, ok);
         else
           flag = lamp_post<D, false, DUMP>(P, g, yw, ktile, P.ks[2], tq, lut, dscr, phi, plo, tscr, lo_dirty,
-                                           st, lam, wc, cks, dump0, grp * kBQ, ph);
+                                           st, lam, wc, cks, dump0, grp * kBQ, ph, &bars[kPvDone], (n - 1) & 1, n > 0,
+                                           status, ok);
       } else {
-        // no visible pair for this group: its rows of the P tile are zero
+        // no visible pair for this group: its rows of the P tile are zero (once the previous
+        // P V product has read them)
+        if (n > 0) ok = ok && ptx::mbar_wait(&bars[kPvDone], (n - 1) & 1, status, kTimeoutCode);
+        ptx::tc_fence_after();
         for (int c = lane; c < kBQ * 8; c += 32) {
           *reinterpret_cast<uint4*>(phi + sw128(grp * kBQ + (c >> 3), c & 7)) = make_uint4(0, 0, 0, 0);
           if (lo_dirty) *reinterpret_cast<uint4*>(plo + sw128(grp * kBQ + (c >> 3), c & 7)) = make_uint4(0, 0, 0, 0);
