@@ -55,8 +55,12 @@ enum Bar {
   kKbfFull = 0, kKbfEmpty,
   // fp32 K half-tile m lives in buffer m & 1 and is announced on barrier m & 3: a compute warp
   // only meets every other tile, and must never be two completions behind on a barrier it polls
-  kKfFull0, kKfEmpty0 = kKfFull0 + 4, kVFull = kKfEmpty0 + 4, kVHalf, kPReady, kPvDone,
-  kSlotFull0,                              // [group][slot]: a packed chain tile waits in TMEM
+  kKfFull0, kKfEmpty0 = kKfFull0 + 4, kVFull = kKfEmpty0 + 4,
+  kVFree,                // every MMA that reads the V buffer has completed
+  kPReady0,              // [group]: the group's 32 rows of the P tile are written
+  kPvDone0 = kPReady0 + 4,   // [group]: the group's P V product (its 32 TMEM lanes) has completed
+  kSlotPad = kPvDone0 + 4,
+  kSlotFull0 = kSlotPad,                   // [group][slot]: a packed chain tile waits in TMEM
   kSlotEmpty0 = kSlotFull0 + 4 * kSlots,   // [group][slot]: the decision-path warp has taken it
   kNumBars = kSlotEmpty0 + 4 * kSlots
 };
@@ -689,7 +693,7 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
   double* dscr_all = reinterpret_cast<double*>(smem + L::kDscr);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBar);
   uint32_t* tslot = reinterpret_cast<uint32_t*>(smem + L::kMisc);
-  uint32_t* lomask = tslot + 1;   // [2]
+  uint32_t* lomask = tslot + 1;   // [group][tile parity]
   int* status = &gstats->status;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -715,12 +719,14 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
       ptx::mbar_init(&bars[kKfEmpty0 + i], 4);
     }
     ptx::mbar_init(&bars[kVFull], 1);
-    ptx::mbar_init(&bars[kVHalf], 1);
-    ptx::mbar_init(&bars[kPReady], 4);
-    ptx::mbar_init(&bars[kPvDone], 1);
+    ptx::mbar_init(&bars[kVFree], 1);
+    for (int i = 0; i < 4; ++i) {
+      ptx::mbar_init(&bars[kPReady0 + i], 1);
+      ptx::mbar_init(&bars[kPvDone0 + i], 1);
+    }
     for (int i = 0; i < 8 * kSlots; ++i) ptx::mbar_init(&bars[kSlotFull0 + i], 1);
     ptx::fence_barrier_init();
-    lomask[0] = lomask[1] = 0;
+    for (int i = 0; i < 8; ++i) lomask[i] = 0;
   }
   if (warp == kCtrlWarp) {
     ptx::tmem_alloc(tslot, 512);
@@ -789,33 +795,53 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
       };
       if (lane == 0) load_v(0);
       __syncwarp();
+      // Each group's rows are multiplied on their own (the MMA writes only that group's 32 TMEM
+      // lanes), as soon as that group has delivered its part of the P tile: the decision paths of
+      // the four groups take very different times per tile and must not wait for one another.
+      int nv = 0;   // V half-tiles consumed
       for (int n = 0; n < T && ok; ++n) {
-        ok = ptx::mbar_wait(&bars[kPReady], n & 1, status, kTimeoutCode);
-        uint32_t lom = 0;
 #pragma unroll 1
         for (int hh = 0; hh < NH && ok; ++hh) {
           const int mv = n * NH + hh;
           ok = ptx::mbar_wait(&bars[kVFull], mv & 1, status, kTimeoutCode);
-          ok = __all_sync(kFull, ok);
-          ptx::tc_fence_after();
-          if (lane == 0 && ok) {
-            if (hh == 0) { lom = lomask[n & 1]; lomask[n & 1] = 0; }
+          uint32_t served = 0;
+          for (uint32_t spin = 0; served != 0xfu && ok; ++spin) {
+#pragma unroll 1
+            for (int g = 0; g < 4; ++g) {
+              if ((served >> g) & 1u) continue;
+              bool ready = hh > 0 || ptx::mbar_try_wait(&bars[kPReady0 + g], n & 1);
+              ready = __shfl_sync(kFull, (int)ready, 0) != 0;   // one answer for the whole warp
+              if (!ready) continue;
+              served |= 1u << g;
+              ptx::tc_fence_after();
+              if (lane == 0) {
+                const uint32_t lom = lomask[2 * g + (n & 1)];
 #pragma unroll
-            for (int ks = 0; ks < 4; ++ks) {
-              const uint64_t bd = ptx::smem_desc_sw128(ptx::smem_u32(vs) + ks * 2048, 8192, 1024);
-              ptx::umma_bf16(tbase + kHalf * hh, ptx::smem_desc_sw128(ptx::smem_u32(phi) + ks * 32, 16, 1024), bd,
-                             idesc, (n > 0 || ks > 0) ? 1u : 0u);
-              if ((lom >> ks) & 1u)
-                ptx::umma_bf16(tbase + kHalf * hh, ptx::smem_desc_sw128(ptx::smem_u32(plo) + ks * 32, 16, 1024), bd,
-                               idesc, 1u);
+                for (int ks = 0; ks < 4; ++ks) {
+                  const uint64_t bd = ptx::smem_desc_sw128(ptx::smem_u32(vs) + ks * 2048, 8192, 1024);
+                  ptx::umma_bf16_lanes(tbase + kHalf * hh, ptx::smem_desc_sw128(ptx::smem_u32(phi) + ks * 32, 16, 1024),
+                                       bd, idesc, (n > 0 || ks > 0) ? 1u : 0u, g);
+                  if ((lom >> ks) & 1u)
+                    ptx::umma_bf16_lanes(tbase + kHalf * hh, ptx::smem_desc_sw128(ptx::smem_u32(plo) + ks * 32, 16, 1024),
+                                         bd, idesc, 1u, g);
+                }
+                if (hh + 1 == NH) ptx::umma_commit(&bars[kPvDone0 + g]);
+              }
+              __syncwarp();
             }
-            ptx::umma_commit(hh + 1 < NH ? &bars[kVHalf] : &bars[kPvDone]);
+            if (served != 0xfu) {
+              if (spin > ptx::kSpinLimit) { atomicExch(status, kTimeoutCode); ok = false; }
+              else if (spin > 64) __nanosleep(64);
+            }
           }
-          __syncwarp();
-          // the V buffer is single: the next half-tile may land once these MMAs have read it
+          ok = __all_sync(kFull, ok);
+          // the V buffer is single: the next half-tile may land once all these MMAs have read it
           if (mv + 1 < M && ok) {
-            ok = ptx::mbar_wait(hh + 1 < NH ? &bars[kVHalf] : &bars[kPvDone], n & 1, status, kTimeoutCode);
+            if (lane == 0) ptx::umma_commit(&bars[kVFree]);
+            __syncwarp();
+            ok = ptx::mbar_wait(&bars[kVFree], nv & 1, status, kTimeoutCode);
             if (lane == 0 && ok) load_v(mv + 1);
+            ++nv;
           }
           ok = __all_sync(kFull, ok);
         }
@@ -957,16 +983,16 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
         const __nv_bfloat16* ktile = kg + (int64_t)i0 * P.ks[2];
         if (full)
           flag = lamp_post<D, true, DUMP>(P, g, yw, ktile, P.ks[2], tq, lut, dscr, phi, plo, tscr, lo_dirty,
-                                          st, lam, wc, cks, dump0, grp * kBQ, ph, &bars[kPvDone], (n - 1) & 1, n > 0,
+                                          st, lam, wc, cks, dump0, grp * kBQ, ph, &bars[kPvDone0 + grp], (n - 1) & 1, n > 0,
                                           status, ok);
         else
           flag = lamp_post<D, false, DUMP>(P, g, yw, ktile, P.ks[2], tq, lut, dscr, phi, plo, tscr, lo_dirty,
-                                           st, lam, wc, cks, dump0, grp * kBQ, ph, &bars[kPvDone], (n - 1) & 1, n > 0,
+                                           st, lam, wc, cks, dump0, grp * kBQ, ph, &bars[kPvDone0 + grp], (n - 1) & 1, n > 0,
                                            status, ok);
       } else {
         // no visible pair for this group: its rows of the P tile are zero (once the previous
         // P V product has read them)
-        if (n > 0) ok = ok && ptx::mbar_wait(&bars[kPvDone], (n - 1) & 1, status, kTimeoutCode);
+        if (n > 0) ok = ok && ptx::mbar_wait(&bars[kPvDone0 + grp], (n - 1) & 1, status, kTimeoutCode);
         ptx::tc_fence_after();
         for (int c = lane; c < kBQ * 8; c += 32) {
           *reinterpret_cast<uint4*>(phi + sw128(grp * kBQ + (c >> 3), c & 7)) = make_uint4(0, 0, 0, 0);
@@ -998,11 +1024,11 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
         ptx::tmem_wait_st();
       }
       const uint32_t lo_now = (flag | (flag >> 4)) & 15u;
-      if (lane == 0 && lo_now) atomicOr(&lomask[n & 1], lo_now);
+      if (lane == 0) lomask[2 * grp + (n & 1)] = lo_now;
       ptx::fence_proxy_async();
       ptx::tc_fence_before();
       __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(&bars[kPReady]);
+      if (lane == 0) ptx::mbar_arrive(&bars[kPReady0 + grp]);
       LAMP_TOC(7, t_r);
 
       const int64_t gt = (((int64_t)b * P.heads_q + h) * (P.seqlen / kBQ) + (j0 / kBQ)) * ntk + t;
@@ -1018,7 +1044,7 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
     }
 
     // ---- epilogue: O / omega, lse = mu + ln(omega) --------------------------------------------------
-    ok = ok && ptx::mbar_wait(&bars[kPvDone], (T - 1) & 1, status, kTimeoutCode);
+    ok = ok && ptx::mbar_wait(&bars[kPvDone0 + grp], (T - 1) & 1, status, kTimeoutCode);
     ptx::tc_fence_after();
     float om_row = st.om[0], mu_row = st.mu[0];   // row = lane = 4*qa + (lane & 3)
 #pragma unroll
