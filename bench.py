@@ -274,7 +274,7 @@ def main():
     peak = 4.0 / MIN_SLOTS_PER_STEP * SM_COUNT * LANES_PER_SM * SM_MAX_MHZ * 1e6 / 1e12
     # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu capture summarised in
     # profiles/lamp_fwd_sm100_config2_ncu_full.txt (algorithmic bytes: 680 MB)
-    traffic = {2: 658.75e6}.get(cfg.index) if args.mode == "lamp" else None
+    traffic = {2: 659.69e6}.get(cfg.index) if args.mode == "lamp" else None
     roofline = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                 "frac": achieved / peak, "traffic": traffic,
                 "note": "peak = issue-slot bound of the emulated e4m3 accumulation at 2 slots/step, "
