@@ -153,6 +153,13 @@ int lamp_attn_fwd_digest(const void* q, const void* k, const void* v, void* out,
                          uint8_t* flag_mask, const lamp_attn_params* p, uint64_t* digest,
                          void* cuda_stream);
 
+/* Test hook: apply the kernel's e4m3 rounding (the operation behind every step of the
+ * low-precision accumulation of Sec. 3.3 / Sec. 4.1: round-to-nearest-even onto the e4m3 grid
+ * with subnormals, saturating at +-448) to n fp32 values.
+ *   in, out  device, n floats each (may alias)
+ * Inputs must be finite with |x| < 2^100.  Asynchronous on the stream. */
+int lamp_attn_debug_round_e4m3(const float* in, float* out, size_t n, void* cuda_stream);
+
 /* Wait for the stream, then copy the counters of the last lamp_attn_fwd on the current
  * device to *host_out.  Returns LAMP_ERR_DEVICE_TIMEOUT if that kernel gave up a wait. */
 int lamp_attn_get_stats(lamp_attn_stats* host_out, void* cuda_stream);

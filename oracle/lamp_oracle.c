@@ -503,6 +503,12 @@ int lamp_oracle_units(const uint16_t* q, const uint16_t* k, const uint16_t* v,
   return 0;
 }
 
+/* The rounding of Sec. 3.3 over an array (for checking a device's rounding routine in bulk). */
+void lamp_oracle_rne_e4m3_array(const float* in, float* out, int64_t n) {
+#pragma omp parallel for schedule(static)
+  for (int64_t i = 0; i < n; ++i) out[i] = lamp_oracle_rne_e4m3(in[i]);
+}
+
 /* One low-precision dot product on its own (for the accumulation-order pins):
  * c <- RNE_e4m3(fmaf(a[t], b[t], c)), t ascending, c0 = +0. */
 float lamp_oracle_chain8(const float* a, const float* b, int n) {

@@ -70,10 +70,20 @@ def lib():
         L.lamp_oracle_stage2.argtypes = [C.c_void_p, C.c_void_p, f32, u32]
         L.lamp_oracle_chain8.restype = f32
         L.lamp_oracle_chain8.argtypes = [C.c_void_p, C.c_void_p, C.c_int]
+        L.lamp_oracle_rne_e4m3_array.restype = None
+        L.lamp_oracle_rne_e4m3_array.argtypes = [C.c_void_p, C.c_void_p, C.c_int64]
         L.lamp_oracle_units.restype = C.c_int
         L.lamp_oracle_units.argtypes = [C.c_void_p] * 3 + [C.POINTER(Params), C.c_int64] + [C.c_void_p] * 7 + [C.POINTER(Stats)]
         _lib = L
     return _lib
+
+
+def rne_e4m3_array(x: np.ndarray) -> np.ndarray:
+    """The oracle's e4m3 rounding, element by element, on a float32 array."""
+    x = np.ascontiguousarray(x, np.float32)
+    out = np.empty_like(x)
+    lib().lamp_oracle_rne_e4m3_array(x.ctypes.data_as(C.c_void_p), out.ctypes.data_as(C.c_void_p), x.size)
+    return out
 
 
 @dataclass

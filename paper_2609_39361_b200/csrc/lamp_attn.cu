@@ -251,6 +251,15 @@ int lamp_attn_fwd(const void* q, const void* k, const void* v, void* out, float*
 // lamp_attn_fwd_digest: the checksum buffer of the forward kernel lives in the library image.
 namespace lamp {
 
+__global__ void lamp_round_e4m3_kernel(const float* __restrict__ in, float* __restrict__ out, size_t n) {
+  for (size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 2; i < n; i += (size_t)gridDim.x * blockDim.x * 2) {
+    float a = in[i], b = i + 1 < n ? in[i + 1] : 0.0f;
+    rne_e4m3_x2(a, b);   // the pairwise conversion-unit rounding the chain uses
+    out[i] = a;
+    if (i + 1 < n) out[i + 1] = b;
+  }
+}
+
 // Scratch of the digest call: two 64-bit checksums per (group, key tile) pair.  Device code may
 // name the array; host code may not use the name as a pointer (on the host it is only a handle
 // for cudaGetSymbolAddress).
@@ -311,6 +320,17 @@ int lamp_attn_fwd_digest(const void* q, const void* k, const void* v, void* out,
   lamp_digest_reduce<<<blocks, 256, 0, stream>>>(g_digest_ptr[dev], (size_t)n_pairs,
                                                  (unsigned long long*)digest);
   e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  return LAMP_OK;
+}
+
+int lamp_attn_debug_round_e4m3(const float* in, float* out, size_t n, void* cuda_stream) {
+  if (!in || !out) return LAMP_ERR_INVALID_ARG;
+  if (n == 0) return LAMP_OK;
+  const size_t pairs = (n + 1) / 2;
+  const int blocks = (int)(pairs / 256 + 1 < 4096 ? pairs / 256 + 1 : 4096);
+  lamp_round_e4m3_kernel<<<blocks, 256, 0, (cudaStream_t)cuda_stream>>>(in, out, n);
+  cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
   return LAMP_OK;
 }

@@ -10,6 +10,23 @@ from parity_util import compare_dense_bytes, compare_units, run_gpu
 pytestmark = pytest.mark.gpu
 
 
+def test_rounding_of_the_chain_against_the_oracle_in_bulk():
+    """Every exponent the accumulation can meet times 2^15 mantissas each (all patterns of the top
+    15 mantissa bits: every e4m3 tie and its neighbours), both signs, plus the edges of the grid."""
+    import paper_2609_39361_b200 as lamp
+    exps = np.arange(127 - 40, 127 + 12, dtype=np.uint32)                 # 2^-40 .. 2^11
+    mant = (np.arange(1 << 15, dtype=np.uint32) << 8)
+    bits = ((exps[:, None] << 23) | mant[None, :]).reshape(-1)
+    bits = np.concatenate([bits, bits | 0x80000000, bits | 0x7f, (bits | 0x80) - 1,
+                           np.array([0, 0x80000000, 0x43e00000, 0x43e80000, 0x43e7ffff], np.uint32)])
+    x = bits.view(np.float32)
+    got = lamp.lamp_attn_debug_round_e4m3(torch.from_numpy(x).cuda()).cpu().numpy()
+    want = oracle.rne_e4m3_array(x)
+    assert np.array_equal(got, want)          # values (and -0 == +0)
+    nz = want != 0
+    assert np.array_equal(np.signbit(got[nz]), np.signbit(want[nz]))
+
+
 def test_config0_dense():
     cfg = li.CONFIGS[0]
     q, k, v = li.make_qkv(cfg)
