@@ -138,16 +138,20 @@ __device__ __forceinline__ void chain8(const void* __restrict__ q, const float* 
 
 // 16-bit logits of one sub-block for this lane's (quad x 4 keys): a sequential fp64 fma
 // chain over kk, scaled, rounded once to e4m11, stored to TMEM columns tdst..tdst+15.
-// The fp32 -> fp64 conversions are the slow part on this GPU, so the warp converts each
-// operand once per 8 channels into a small shared-memory scratch (16 keys and 32 rows as
-// doubles) and every lane reads from there.
-// krow: global bf16 row of the sub-block's first key (lanes 0-15 fetch key `lane`, 16 bytes
-// per 8 channels; the rows were just streamed through L2 by TMA); tq: TMEM columns holding
-// the raw bf16 query row of this lane (row = lane of the group), two channels per column;
-// dscr: 384 doubles for the warp.
+// The fp32 -> fp64 conversions are the slow part on this GPU (they hold the scheduler for
+// several cycles each), so the warp converts each operand once per 8 channels into a small
+// shared-memory scratch (16 keys and 32 rows as doubles) and every lane reads from there.
+// krow: global bf16 row of the sub-block's first key (lane l fetches key l % 16, channels
+// 4 (l / 16) .. +3 of every 8; the rows were just streamed through L2 by TMA).
+// tq: TMEM columns holding the query row of this lane (row = lane of the group).  head_dim 128:
+// one column per channel, the high word of the channel as a double (the low word of a widened
+// bf16 is zero), converted once per CTA; head_dim 256: raw bf16, two channels per column, converted
+// here.  dscr: 384 doubles for the warp.
 template <int D>
 __device__ __noinline__ void dot16(const __nv_bfloat16* __restrict__ krow, int64_t kstride, uint32_t tq,
                                    double* dscr, double scale_d, uint32_t tdst) {
+  constexpr bool QHI = (D == 128);
+  constexpr int QW = QHI ? 8 : 4;   // TMEM columns per 8 channels
   const int lane = threadIdx.x & 31, qa = lane >> 2, tp = lane & 3;
   __builtin_assume(__isShared(dscr));
   double* kscr = dscr;          // [8 kk][16 keys]
@@ -157,25 +161,39 @@ __device__ __noinline__ void dot16(const __nv_bfloat16* __restrict__ krow, int64
   for (int a = 0; a < 4; ++a)
 #pragma unroll
     for (int b = 0; b < 4; ++b) acc[a][b] = 0.0;
-  const __nv_bfloat16* ksrc = krow + (int64_t)(lane & 15) * kstride;
-  uint4 kraw = *reinterpret_cast<const uint4*>(ksrc);
-  uint4 qraw;
-  ptx::tmem_ld4(tq, qraw);
+  const int kh = lane >> 4;      // which four of a chunk's eight channels this lane converts for K
+  const __nv_bfloat16* ksrc = krow + (int64_t)(lane & 15) * kstride + 4 * kh;
+  uint2 kraw = *reinterpret_cast<const uint2*>(ksrc);
+  uint32_t qraw[QW];
+  auto fetch_q = [&](int k0) {
+    if constexpr (QHI) {
+      ptx::tmem_ld8(tq + k0, qraw);
+    } else {
+      uint4 v;
+      ptx::tmem_ld4(tq + (k0 >> 1), v);
+      qraw[0] = v.x; qraw[1] = v.y; qraw[2] = v.z; qraw[3] = v.w;
+    }
+  };
+  fetch_q(0);
   ptx::tmem_wait_ld();
 #pragma unroll 1
   for (int k0 = 0; k0 < D; k0 += 8) {
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
-      const uint32_t wq = (&qraw.x)[e >> 1];
-      qscr[e * 32 + lane] = (double)__uint_as_float((e & 1) ? (wq & 0xffff0000u) : (wq << 16));
-      if (lane < 16) {
-        const uint32_t wk = (&kraw.x)[e >> 1];
-        kscr[e * 16 + lane] = (double)__uint_as_float((e & 1) ? (wk & 0xffff0000u) : (wk << 16));
+      if constexpr (QHI) {
+        qscr[e * 32 + lane] = __hiloint2double((int)qraw[e], 0);
+      } else {
+        const uint32_t wq = qraw[e >> 1];
+        qscr[e * 32 + lane] = (double)__uint_as_float((e & 1) ? (wq & 0xffff0000u) : (wq << 16));
+      }
+      if (e < 4) {
+        const uint32_t wk = (e >> 1) ? kraw.y : kraw.x;
+        kscr[(4 * kh + e) * 16 + (lane & 15)] = (double)__uint_as_float((e & 1) ? (wk & 0xffff0000u) : (wk << 16));
       }
     }
     const int kn = (k0 + 8) & (D - 1);      // next chunk's operands travel while this one is used
-    kraw = *reinterpret_cast<const uint4*>(ksrc + kn);
-    ptx::tmem_ld4(tq + (kn >> 1), qraw);
+    kraw = *reinterpret_cast<const uint2*>(ksrc + kn);
+    fetch_q(kn);
     __syncwarp();
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
@@ -760,9 +778,10 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tbase = *tslot;
-  // TMEM columns of a group's lanes: [0, D) O, 64 for the 16-bit logits, D/2 for the lane's raw bf16
-  // query row (operand of the 16-bit dots), kSlots x 16 for the ring of packed first-pass logits
-  constexpr uint32_t kColScr = D, kColQ = D + 64, kColRing = D + 64 + D / 2;
+  // TMEM columns of a group's lanes: [0, D) O; 64 for the 16-bit logits; 128 for the lane's query row
+  // as operand of the 16-bit dots (head_dim 128: the high word of each channel as a double, head_dim
+  // 256: raw bf16 pairs); kSlots x 16 for the ring of packed first-pass logits
+  constexpr uint32_t kColScr = D, kColQ = D + 64, kColRing = D + 64 + 128;
   static_assert(kColRing + 16 * kSlots <= 512, "TMEM columns");
 
   if (warp >= 12) {
@@ -931,12 +950,21 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
     {
       const __nv_bfloat16* qrow = P.q + b * P.qs[0] + h * P.qs[1] + (int64_t)(j0 + lane) * P.qs[2];
 #pragma unroll 1
-      for (int c0 = 0; c0 < D / 2; c0 += 16) {
+      for (int c0 = 0; c0 < 128; c0 += 16) {
         uint32_t r[16];
+        if (D == 128) {   // 16 channels, widened to double here, once: the high words
+          const uint4 v0 = *reinterpret_cast<const uint4*>(qrow + c0);
+          const uint4 v1 = *reinterpret_cast<const uint4*>(qrow + c0 + 8);
+          const uint32_t w[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const uint4 v = *reinterpret_cast<const uint4*>(qrow + 2 * c0 + 8 * i);
-          r[4 * i] = v.x; r[4 * i + 1] = v.y; r[4 * i + 2] = v.z; r[4 * i + 3] = v.w;
+          for (int i = 0; i < 16; ++i)
+            r[i] = (uint32_t)__double2hiint((double)__uint_as_float((i & 1) ? (w[i >> 1] & 0xffff0000u) : (w[i >> 1] << 16)));
+        } else {          // 32 channels, raw
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const uint4 v = *reinterpret_cast<const uint4*>(qrow + 2 * c0 + 8 * i);
+            r[4 * i] = v.x; r[4 * i + 1] = v.y; r[4 * i + 2] = v.z; r[4 * i + 3] = v.w;
+          }
         }
         ptx::tmem_st16(tq + c0, r);
       }
