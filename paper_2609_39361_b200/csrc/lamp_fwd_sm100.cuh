@@ -156,6 +156,8 @@ __device__ __noinline__ void dot16(const __nv_bfloat16* __restrict__ krow, int64
   __builtin_assume(__isShared(dscr));
   double* kscr = dscr;          // [8 kk][16 keys]
   double* qscr = dscr + 128;    // [8 kk][32 rows]
+  uint32_t* khi = reinterpret_cast<uint32_t*>(kscr) + 1;   // high words of the same
+  uint32_t* qhi = reinterpret_cast<uint32_t*>(qscr) + 1;
   double acc[4][4];
 #pragma unroll
   for (int a = 0; a < 4; ++a)
@@ -180,15 +182,18 @@ __device__ __noinline__ void dot16(const __nv_bfloat16* __restrict__ krow, int64
   for (int k0 = 0; k0 < D; k0 += 8) {
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
+      // a widened bf16 has a zero low word: only the high words are ever written, the low
+      // words of the scratch were cleared when the kernel started
       if constexpr (QHI) {
-        qscr[e * 32 + lane] = __hiloint2double((int)qraw[e], 0);
+        qhi[2 * (e * 32 + lane)] = qraw[e];
       } else {
         const uint32_t wq = qraw[e >> 1];
-        qscr[e * 32 + lane] = (double)__uint_as_float((e & 1) ? (wq & 0xffff0000u) : (wq << 16));
+        qhi[2 * (e * 32 + lane)] = (uint32_t)__double2hiint((double)__uint_as_float((e & 1) ? (wq & 0xffff0000u) : (wq << 16)));
       }
       if (e < 4) {
         const uint32_t wk = (e >> 1) ? kraw.y : kraw.x;
-        kscr[(4 * kh + e) * 16 + (lane & 15)] = (double)__uint_as_float((e & 1) ? (wk & 0xffff0000u) : (wk << 16));
+        khi[2 * ((4 * kh + e) * 16 + (lane & 15))] =
+            (uint32_t)__double2hiint((double)__uint_as_float((e & 1) ? (wk & 0xffff0000u) : (wk << 16)));
       }
     }
     const int kn = (k0 + 8) & (D - 1);      // next chunk's operands travel while this one is used
@@ -752,6 +757,7 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
     if (lane == 0) { ptx::prefetch_tensormap(&kmap); ptx::prefetch_tensormap(&vmap); }
   }
   for (int i = tid; i < 128; i += kThreads) lut[i] = lut_g[i];
+  for (int i = tid; i < 4 * 384; i += kThreads) dscr_all[i] = 0.0;
   {
     const __nv_bfloat16* qg = P.q + b * P.qs[0] + h * P.qs[1] + (int64_t)m0 * P.qs[2];
     for (int c = tid; c < kBM * D / 8; c += kThreads) {
