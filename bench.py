@@ -6,6 +6,12 @@ One "step" is one forward pass (the whole hot path: emulated 8-bit logits, flagg
 input (B=4, 32 query / 8 KV heads, N=8192, head_dim 128, causal).  Prints ONE JSON line.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config C]
+                  [--mode lamp|force8|force16] [--tau T] [--delta D] [--no-stage1]
+                  [--scale-mult M] [--window W]
+
+The options after --config select the other workloads and the paper's ablations (threshold
+and margin sweeps, stage 1 off, the scale sweep of the long-context config, the sliding
+window of the Gemma-shaped config); without them the line is the headline configuration.
 
 With N > 1 (under torchrun) every rank runs the same workload on its own GPU: units
 (batch, head, 32-row group) are independent, so there is no data-path collective
@@ -16,6 +22,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -117,14 +124,23 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
-def oracle_sample_run(cfg, q, k, v, scale, n_units, seed=11):
+def oracle_sample_run(cfg, q, k, v, scale, n_units, seed=11, knobs=None):
     import oracle
+    kn = knobs or {}
+    window = kn.get("window", 0)
     units = li.sample_units(cfg, n_units, seed=seed)
     t0 = time.perf_counter()
-    oracle.run_units(q, k, v, units, scale=scale, causal=cfg.causal, checksums=False)
+    oracle.run_units(q, k, v, units, scale=scale, causal=cfg.causal, window=window, tau=kn.get("tau", 0.5),
+                     delta=kn.get("delta", 2.0 ** -8), flags=kn.get("flags", 0), checksums=False)
     dt = time.perf_counter() - t0
-    fl = sum(4.0 * cfg.D * unit_pairs(cfg, int(g)) for _, _, g in units)
+    fl = sum(4.0 * cfg.D * unit_pairs(cfg, int(g), window) for _, _, g in units)
     return dt, fl, len(units)
+
+
+def knobs_of(args):
+    """Thresholds, mode bits and mask of this run (the same numeric flag values in the library and the oracle)."""
+    flags = {"lamp": 0, "force8": 2, "force16": 1}[args.mode] | (4 if args.no_stage1 else 0)
+    return {"tau": args.tau, "delta": args.delta, "flags": flags, "window": args.window}
 
 
 def reference_arm(args, cfg, rank):
@@ -134,16 +150,17 @@ def reference_arm(args, cfg, rank):
     import oracle
     oracle.build()
     q, k, v = li.make_qkv(cfg)
-    scale = li.softmax_scale(cfg.D)
+    scale = li.softmax_scale(cfg.D, args.scale_mult)
+    kn = knobs_of(args)
     cores = os.cpu_count() or 1
-    dt, fl, n = oracle_sample_run(cfg, q, k, v, scale, max(8, cores))      # calibration
+    dt, fl, n = oracle_sample_run(cfg, q, k, v, scale, max(8, cores), knobs=kn)      # calibration
     per_unit = dt / n
     n_units = int(max(cores, min(4096, 6.0 / max(per_unit, 1e-6))))
     for _ in range(args.warmup and 1):
-        oracle_sample_run(cfg, q, k, v, scale, n_units)
+        oracle_sample_run(cfg, q, k, v, scale, n_units, knobs=kn)
     tot_t = tot_f = 0.0
     for s in range(args.steps):
-        dt, fl, n = oracle_sample_run(cfg, q, k, v, scale, n_units, seed=100 + s)
+        dt, fl, n = oracle_sample_run(cfg, q, k, v, scale, n_units, seed=100 + s, knobs=kn)
         tot_t += dt; tot_f += fl
     val = tot_f / tot_t / 1e12
     sample = f"{n_units} of {cfg.B * cfg.Hq * cfg.N // 32} (b, h, 32-row group) units per step, seeded spread"
@@ -151,15 +168,22 @@ def reference_arm(args, cfg, rank):
             "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": 1e3 * tot_t / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "e4m3-emulated/f32", "data": "synthetic",
-            "config": workload_config(cfg),
+            "config": workload_config(cfg, args),
             "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
 
 
-def workload_config(cfg):
+def workload_config(cfg, args):
+    extra = ""
+    if args.window:
+        extra += f", window={args.window}"
+    if args.scale_mult != 1.0:
+        extra += f", scale x{args.scale_mult:g}"
+    if args.no_stage1:
+        extra += ", stage 1 off"
     return {"workload": f"config {cfg.index}: {cfg.name} prefill, B={cfg.B}, Hq={cfg.Hq}, Hkv={cfg.Hkv}, "
-                        f"N={cfg.N}, head_dim={cfg.D}, causal, tau=0.5, delta=2^-8",
+                        f"N={cfg.N}, head_dim={cfg.D}, causal{extra}, tau={args.tau:g}, delta=2^{math.log2(args.delta):g}",
             "l2": "inputs (Q+K+V+O = %.0f MB) larger than the 126 MB L2" %
                   ((2 * cfg.B * cfg.Hq + 2 * cfg.B * cfg.Hkv) * cfg.N * cfg.D * 2 / 1e6)}
 
@@ -174,6 +198,11 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--mode", default="lamp", choices=["lamp", "force8", "force16"],
                     help="internal comparison modes: pure 8-bit / every sub-block 16-bit")
+    ap.add_argument("--tau", type=float, default=0.5, help="threshold of eq. (8)")
+    ap.add_argument("--delta", type=float, default=2.0 ** -8, help="safety margin of eq. (7)")
+    ap.add_argument("--no-stage1", action="store_true", help="the ablation without the running-maximum test")
+    ap.add_argument("--scale-mult", type=float, default=1.0, help="softmax scale = mult / sqrt(head_dim)")
+    ap.add_argument("--window", type=int, default=0, help="sliding window (0 = global causal)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -200,7 +229,8 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    scale = li.softmax_scale(cfg.D)
+    scale = li.softmax_scale(cfg.D, args.scale_mult)
+    kn = knobs_of(args)
     q, k, v = li.make_qkv(cfg)
     hq, hk, hv = q.pin_memory(), k.pin_memory(), v.pin_memory()
     dq, dk, dv = hq.to(dev), hk.to(dev), hv.to(dev)
@@ -211,9 +241,9 @@ def main():
     p = lamp.lamp_attn_default_params()
     p.batch, p.heads_q, p.heads_kv, p.seqlen, p.head_dim = B, Hq, k.shape[1], N, D
     lamp.lamp_attn_contiguous_strides(p)
-    p.causal, p.scale = 1, scale
-    p.flags = {"lamp": 0, "force8": lamp.LAMP_FORCE_8BIT, "force16": lamp.LAMP_FORCE_16BIT}[args.mode]
-    fl = flops_of(cfg)
+    p.causal, p.window, p.scale = 1, args.window, scale
+    p.threshold, p.delta, p.flags = args.tau, args.delta, kn["flags"]
+    fl = flops_of(cfg, args.window)
 
     def step():
         lamp.lamp_attn_fwd(dq, dk, dv, out, lse, fm, p)
@@ -274,7 +304,9 @@ def main():
     peak = 4.0 / MIN_SLOTS_PER_STEP * SM_COUNT * LANES_PER_SM * SM_MAX_MHZ * 1e6 / 1e12
     # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu capture summarised in
     # profiles/lamp_fwd_sm100_config2_ncu_full.txt (algorithmic bytes: 680 MB)
-    traffic = {2: 659.69e6}.get(cfg.index) if args.mode == "lamp" else None
+    headline = (args.mode == "lamp" and not args.no_stage1 and args.tau == 0.5 and args.delta == 2.0 ** -8
+                and args.scale_mult == 1.0 and args.window == 0)
+    traffic = {2: 659.69e6}.get(cfg.index) if headline else None
     roofline = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                 "frac": achieved / peak, "traffic": traffic,
                 "note": "peak = issue-slot bound of the emulated e4m3 accumulation at 2 slots/step, "
@@ -285,9 +317,9 @@ def main():
         import oracle
         oracle.build()
         cores = os.cpu_count() or 1
-        dt, f1, n = oracle_sample_run(cfg, q, k, v, scale, max(8, cores))
+        dt, f1, n = oracle_sample_run(cfg, q, k, v, scale, max(8, cores), knobs=kn)
         n_units = int(max(cores, min(4096, 15.0 / max(dt / n, 1e-6))))
-        dt, f1, n = oracle_sample_run(cfg, q, k, v, scale, n_units, seed=12)
+        dt, f1, n = oracle_sample_run(cfg, q, k, v, scale, n_units, seed=12, knobs=kn)
         cpu = {"value": f1 / dt / 1e12, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
                "sample": f"{n} of {B * Hq * N // 32} (b, h, 32-row group) units, seeded spread, {dt:.1f} s"}
 
@@ -297,7 +329,7 @@ def main():
     line = {"metric": "lamp_attention_fwd_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world,
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "e4m3-emulated/f32", "data": "synthetic", "config": workload_config(cfg),
+            "dtype": "e4m3-emulated/f32", "data": "synthetic", "config": workload_config(cfg, args),
             "mode": args.mode, "clocks": clk.summary(),
             "e2e": {"value": whole_job_tflops(fl, world, e2e_ms), "unit": "TFLOP/s",
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},

@@ -74,6 +74,20 @@ def test_scale_sweep_saturation(mult):
         compare_units(gpu, ref, check_stats=True, label=f"mult={mult}")
 
 
+@pytest.mark.parametrize("flags,tau,delta", [(0, 0.125, 2.0 ** -8), (0, 0.03125, 2.0 ** -8), (0, 0.5, 2.0 ** -4),
+                                             (oracle.NO_STAGE1, 0.25, 2.0 ** -4), (0, 0.0, 2.0 ** -8)])
+def test_threshold_and_margin_sweeps(flags, tau, delta):
+    """Points of the ablation sweeps (threshold of eq. (8), margin of eq. (7), stage 1 off): where
+    stage 2 does most of the flagging, and tau = 0, which recomputes whatever carries any mass."""
+    cfg = li.CONFIGS[1]
+    q, k, v = li.make_qkv(cfg, Hq=4, Hkv=2, N=512, seed=31)
+    sc = li.softmax_scale(cfg.D)
+    ref = oracle.run_all(q, k, v, scale=sc, tau=tau, delta=delta, flags=flags, dumps=True)
+    gpu = run_gpu(q, k, v, scale=sc, threshold=tau, delta=delta, flags=flags, dump=(0, 1))
+    compare_units(gpu, ref, check_stats=True, label=f"flags={flags} tau={tau} delta={delta}")
+    compare_dense_bytes(gpu, ref, 0, 1)
+
+
 @pytest.mark.parametrize("window,flags", [(0, 0), (192, 0), (0, oracle.FORCE_16BIT)])
 def test_head_dim_256_gemma_shaped(window, flags):
     """head_dim 256 (two 128-channel halves per tile), global and sliding-window layers."""
