@@ -24,7 +24,9 @@
  *     the matrix product is accumulated");
  *   - a warp owns b_q = 32 query rows (Sec. 4.1 gives only b_q N_q = 128);
  *   - 16-bit logits are a sequential fp64 fma chain, rounded once to e4m11;
- *   - among equally small stage-2 recompute sets the smallest bitmask wins.
+ *   - among equally small stage-2 recompute sets the smallest bitmask wins;
+ *   - (optional mode) the compact layout's branch recomputes the remaining 8-bit sub-blocks of a
+ *     tile with two or more marked sub-blocks exactly like stage-2 recomputations.
  * Parity unpinned (no value in the paper fixes them): b_q = 32, the stage-2
  * tie-break, the 16-bit accumulation rounding, the truncated-maximum shift.
  */
@@ -41,6 +43,7 @@
 #define LAMP_FORCE_16BIT 1u
 #define LAMP_FORCE_8BIT  2u
 #define LAMP_NO_STAGE1   4u
+#define LAMP_COMPACT_BRANCH 16u  /* Sec. 3.3 "Register layout": the compact layout's branch (see below) */
 
 typedef struct {
   int32_t batch, heads_q, heads_kv, seqlen, head_dim;
@@ -396,6 +399,11 @@ static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
         }
       Rset = lamp_oracle_stage2(xi, omh, p->tau, freem);
     }
+    /* Compact register layout (Sec. 3.3, "Register layout"): when the two stages mark two or more
+     * sub-blocks of the tile, the update of O falls back to 16 bits for the whole tile.  Reading taken
+     * here: the sub-blocks still held in 8 bits join the stage-2 set and are recomputed under the rule
+     * of Alg. 1's stage-2 recomputation (running maxima unchanged). */
+    if ((p->flags & LAMP_COMPACT_BRANCH) && __builtin_popcount(Theta | Rset) >= 2) Rset = freem;
 
     /* dumps and checksums refer to the 8-bit pass before any stage-2 replacement */
     for (int i = 0; i < TK; ++i)

@@ -18,6 +18,7 @@ _SRC = os.path.join(_HERE, "lamp_oracle.c")
 _SO = os.path.join(_HERE, "liblamp_oracle.so")
 
 FORCE_16BIT, FORCE_8BIT, NO_STAGE1 = 1, 2, 4
+COMPACT_BRANCH = 16   # Sec. 3.3 'Register layout': whole tile to 16 bits once two sub-blocks are marked
 
 
 class Params(C.Structure):

@@ -262,6 +262,39 @@ def test_tau_one_disables_stage_two_and_fraction_is_monotone(small):
         assert ((r.flags[:, 0] & 1) == 1).all()
 
 
+def test_compact_layout_branch(small):
+    """Sec. 3.3 "Register layout": with the compact layout a tile with two or more marked sub-blocks is
+    updated in 16 bits as a whole.  Pins: (1) a tile ends with none, one or all of its active sub-blocks
+    recomputed; (2) up to and including a unit's first such tile the decisions are those of the plain
+    mode, with the rest of that tile moved into the stage-2 set; (3) the result is no further from fp64
+    attention than the plain mode's, and more sub-blocks are recomputed."""
+    q, k, v, sc = small
+    plain = oracle.run_all(q, k, v, scale=sc)
+    comp = oracle.run_all(q, k, v, scale=sc, flags=oracle.COMPACT_BRANCH)
+    N = 512
+    for u, (b, h, g) in enumerate(plain.units):
+        nt = (32 * g + 31) // 64 + 1
+        branched = False
+        for t in range(nt):
+            nact = min(4, (32 * g + 31 - 64 * t) // 16 + 1)          # causal: sub-blocks with a visible pair
+            act = (1 << nact) - 1
+            fc = int(comp.flags[u, t]); pc = bin((fc | fc >> 4) & 15).count("1")
+            assert pc in (0, 1, nact), (u, t, fc)
+            if not branched:
+                fp = int(plain.flags[u, t]); pp = bin((fp | fp >> 4) & 15).count("1")
+                assert (fc & 15) == (fp & 15)
+                if pp >= 2:
+                    assert (fc | fc >> 4) & 15 == act and (fc >> 4) == act & ~(fc & 15)
+                    branched = True
+                else:
+                    assert fc == fp
+    o, _, _ = ref_attention(q, k, v, sc)
+    out_p, _ = dense(plain, 1, 4, N, 128)
+    out_c, _ = dense(comp, 1, 4, N, 128)
+    assert (out_c - o).norm() <= 1.02 * (out_p - o).norm()
+    assert comp.stats["stage1_flagged"] + comp.stats["stage2_flagged"] > plain.stats["stage1_flagged"] + plain.stats["stage2_flagged"]
+
+
 def test_rows_sum_to_one_and_units_are_independent(small):
     q, k, v, sc = small
     ones = torch.ones_like(v)
