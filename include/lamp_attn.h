@@ -43,6 +43,11 @@ typedef enum lamp_attn_error {
 #define LAMP_FORCE_8BIT      0x02u /* no recomputation at all: the paper's pure 8-bit baseline (Sec. 4.1) */
 #define LAMP_NO_STAGE1       0x04u /* skip the running-maximum test (the paper's Appendix D ablation)     */
 #define LAMP_OUT_FP32        0x08u /* `out` is fp32 instead of bf16                                       */
+#define LAMP_COMPACT_BRANCH  0x10u /* the branch of the "compact" register layout (Sec. 3.3, "Register
+                                      layout"): when the two stages mark two or more sub-blocks of a (group,
+                                      key tile), the sub-blocks still held in 8 bits are recomputed too, under
+                                      the rule of stage-2 recomputations (running maxima unchanged); they are
+                                      reported in bits 4-7 of the flag byte and counted in stage2_flagged   */
 
 /* Problem statement of Algorithm 1: Q, K, V per head in HBM, safety margin
  * delta of eq. (7), threshold tau of eq. (8).  Layout: element strides for

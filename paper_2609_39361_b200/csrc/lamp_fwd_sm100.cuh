@@ -631,6 +631,8 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
       if ((r & ~freem) == 0 && ((feas >> r) & 1u) && sz < best) { best = sz; Rset = r; }
     }
   }
+  // compact register layout (Sec. 3.3): two or more marked sub-blocks send the rest of the tile to 16 bits
+  if ((P.flags & LAMP_COMPACT_BRANCH) && __popc(Theta | Rset) >= 2) Rset = freem;
   LAMP_TOC(6, t_s2);
 
   // ---- stage-2 recomputation with the maxima unchanged -------------------------------------------

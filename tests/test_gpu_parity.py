@@ -75,10 +75,14 @@ def test_scale_sweep_saturation(mult):
 
 
 @pytest.mark.parametrize("flags,tau,delta", [(0, 0.125, 2.0 ** -8), (0, 0.03125, 2.0 ** -8), (0, 0.5, 2.0 ** -4),
-                                             (oracle.NO_STAGE1, 0.25, 2.0 ** -4), (0, 0.0, 2.0 ** -8)])
+                                             (oracle.NO_STAGE1, 0.25, 2.0 ** -4), (0, 0.0, 2.0 ** -8),
+                                             (oracle.COMPACT_BRANCH, 0.5, 2.0 ** -8),
+                                             (oracle.COMPACT_BRANCH, 0.125, 2.0 ** -8),
+                                             (oracle.COMPACT_BRANCH | oracle.NO_STAGE1, 0.125, 2.0 ** -8)])
 def test_threshold_and_margin_sweeps(flags, tau, delta):
     """Points of the ablation sweeps (threshold of eq. (8), margin of eq. (7), stage 1 off): where
-    stage 2 does most of the flagging, and tau = 0, which recomputes whatever carries any mass."""
+    stage 2 does most of the flagging, and tau = 0, which recomputes whatever carries any mass; the
+    branch of the compact register layout (Sec. 3.3) on top of them."""
     cfg = li.CONFIGS[1]
     q, k, v = li.make_qkv(cfg, Hq=4, Hkv=2, N=512, seed=31)
     sc = li.softmax_scale(cfg.D)
