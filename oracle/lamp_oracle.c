@@ -23,7 +23,8 @@
  *   - the softmax scale is folded into Q once, in fp32 (Sec. 3.3 "applied before
  *     the matrix product is accumulated");
  *   - a warp owns b_q = 32 query rows (Sec. 4.1 gives only b_q N_q = 128);
- *   - 16-bit logits are a sequential fp64 fma chain, rounded once to e4m11;
+ *   - 16-bit logits are a sequential fp64 fma chain, rounded once to e4m11 (optional mode: the
+ *     per-step e4m11 recursion instead);
  *   - among equally small stage-2 recompute sets the smallest bitmask wins;
  *   - (optional mode) the compact layout's branch recomputes the remaining 8-bit sub-blocks of a
  *     tile with two or more marked sub-blocks exactly like stage-2 recomputations.
@@ -44,6 +45,7 @@
 #define LAMP_FORCE_8BIT  2u
 #define LAMP_NO_STAGE1   4u
 #define LAMP_COMPACT_BRANCH 16u  /* Sec. 3.3 "Register layout": the compact layout's branch (see below) */
+#define LAMP_H16_SEQ     32u     /* 16-bit logits by per-step e4m11 accumulation (the other reading, see logit16) */
 
 typedef struct {
   int32_t batch, heads_q, heads_kv, seqlen, head_dim;
@@ -202,6 +204,27 @@ uint32_t lamp_oracle_stage2(const double xi[NK][BQ], const float* omega_hat, flo
   return free_mask;
 }
 
+float lamp_oracle_chain16(const float* a, const float* b, int n);
+
+/* A 16-bit logit (Alg. 1 "recompute Y_theta in high precision").
+ * Default reading: the exact dot product as a sequential fp64 fma chain over the channels, times the
+ * scale, rounded once to e4m11 (Sec. 3.3 "a 16-bit e4m11 format to accumulate matrix products" taken as
+ * the format of the result).
+ * LAMP_H16_SEQ, the other reading: the same recursion as the 8-bit pass (Sec. 4.1, round(c + a*b) with
+ * the multiplication and addition in fp32), every partial sum rounded to e4m11, on the pre-scaled query. */
+static float logit16(const lamp_oracle_params* p, const uint16_t* krow, const uint16_t* qrow,
+                     const float* qsrow, int D) {
+  if (p->flags & LAMP_H16_SEQ) {
+    float kf[256];
+    for (int kk = 0; kk < D; ++kk) kf[kk] = bf16_to_float(krow[kk]);
+    return lamp_oracle_chain16(kf, qsrow, D);
+  }
+  double acc = 0.0;
+  for (int kk = 0; kk < D; ++kk)
+    acc = fma((double)bf16_to_float(krow[kk]), (double)bf16_to_float(qrow[kk]), acc);
+  return lamp_oracle_rne_e4m11((double)p->scale * acc);
+}
+
 /* ---------------------------------------------------------------- checksum */
 
 static uint64_t mix64(uint64_t x) {
@@ -341,11 +364,7 @@ static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
       for (int i = th * BK; i < (th + 1) * BK; ++i)
         for (int j = 0; j < BQ; ++j) {
           if (!val[i][j]) continue;
-          double acc = 0.0;
-          for (int kk = 0; kk < D; ++kk)
-            acc = fma((double)bf16_to_float(K[(i0 + i) * D + kk]),
-                      (double)bf16_to_float(Q[j * D + kk]), acc);
-          Y16[i][j] = lamp_oracle_rne_e4m11((double)p->scale * acc);
+          Y16[i][j] = logit16(p, K + (size_t)(i0 + i) * D, Q + (size_t)j * D, qs + (size_t)j * D, D);
           if (fabsf(Y16[i][j]) == 448.0f) st->sat_e4m11++;
           if (Y16[i][j] > muh[j]) muh[j] = Y16[i][j];
         }
@@ -425,11 +444,7 @@ static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
       for (int i = th * BK; i < (th + 1) * BK; ++i)
         for (int j = 0; j < BQ; ++j) {
           if (!val[i][j]) continue;
-          double acc = 0.0;
-          for (int kk = 0; kk < D; ++kk)
-            acc = fma((double)bf16_to_float(K[(i0 + i) * D + kk]),
-                      (double)bf16_to_float(Q[j * D + kk]), acc);
-          float y = lamp_oracle_rne_e4m11((double)p->scale * acc);
+          float y = logit16(p, K + (size_t)(i0 + i) * D, Q + (size_t)j * D, qs + (size_t)j * D, D);
           if (fabsf(y) == 448.0f) st->sat_e4m11++;
           float d = y - muh[j];
           Ef[i][j] = lamp_oracle_exp16((float)rne_sig((double)d, 12));
@@ -515,6 +530,14 @@ int lamp_oracle_units(const uint16_t* q, const uint16_t* k, const uint16_t* v,
 void lamp_oracle_rne_e4m3_array(const float* in, float* out, int64_t n) {
 #pragma omp parallel for schedule(static)
   for (int64_t i = 0; i < n; ++i) out[i] = lamp_oracle_rne_e4m3(in[i]);
+}
+
+/* The same recursion on the 16-bit grid: c <- RNE_e4m11(fmaf(a[t], b[t], c)), t ascending, c0 = +0
+ * (the fp32 result of the fused multiply-add is exact in double, so one rounding follows it). */
+float lamp_oracle_chain16(const float* a, const float* b, int n) {
+  float c = 0.0f;
+  for (int t = 0; t < n; ++t) c = lamp_oracle_rne_e4m11((double)fmaf(a[t], b[t], c));
+  return c;
 }
 
 /* One low-precision dot product on its own (for the accumulation-order pins):

@@ -18,6 +18,7 @@ _SRC = os.path.join(_HERE, "lamp_oracle.c")
 _SO = os.path.join(_HERE, "liblamp_oracle.so")
 
 FORCE_16BIT, FORCE_8BIT, NO_STAGE1 = 1, 2, 4
+H16_SEQ = 32          # 16-bit logits by per-step e4m11 accumulation (Sec. 4.1 recursion) instead of one rounding
 COMPACT_BRANCH = 16   # Sec. 3.3 'Register layout': whole tile to 16 bits once two sub-blocks are marked
 
 
@@ -69,6 +70,8 @@ def lib():
         L.lamp_oracle_exp16.restype = f32; L.lamp_oracle_exp16.argtypes = [f32]
         L.lamp_oracle_stage2.restype = u32
         L.lamp_oracle_stage2.argtypes = [C.c_void_p, C.c_void_p, f32, u32]
+        L.lamp_oracle_chain16.restype = f32
+        L.lamp_oracle_chain16.argtypes = [C.c_void_p, C.c_void_p, C.c_int]
         L.lamp_oracle_chain8.restype = f32
         L.lamp_oracle_chain8.argtypes = [C.c_void_p, C.c_void_p, C.c_int]
         L.lamp_oracle_rne_e4m3_array.restype = None

@@ -101,6 +101,47 @@ def test_chain_swamping_examples():
         float(np.float32(np.float64(np.float32(1.4375)) * 3.0 + 0.3125)))
 
 
+def chain16(a, b):
+    a = np.asarray(a, np.float32); b = np.asarray(b, np.float32)
+    return L.lamp_oracle_chain16(a.ctypes.data_as(C.c_void_p), b.ctypes.data_as(C.c_void_p), len(a))
+
+
+def test_per_step_e4m11_recursion_examples():
+    """The other reading of the 16-bit accumulation: round(c + a*b) onto e4m11 at every step (Sec. 4.1).
+    Values worked by hand on the 12-significant-bit grid."""
+    assert chain16([1.0] * 128, [1.0] * 128) == 128.0                 # integers below 4096 are exact
+    assert chain16([1.0] + [2.0 ** -13] * 100, [1.0] * 101) == 1.0      # a quarter ulp of 1.0 is swallowed every time
+    assert chain16([2.0 ** -13] * 100 + [1.0], [1.0] * 101) == float(np.float32(1.0 + 100 * 2.0 ** -13))
+    assert chain16([1.0, 2.0 ** -12], [1.0, 1.0]) == 1.0                # tie (half an ulp) goes to the even neighbour
+    assert chain16([1.0 + 2.0 ** -11, 2.0 ** -12], [1.0, 1.0]) == 1.0 + 2.0 ** -10
+    assert chain16([300.0, 300.0], [1.0, 1.0]) == 448.0                 # saturation
+    assert chain16([-300.0, -300.0, 1.0], [1.0, 1.0, 1.0]) == -447.0
+    assert chain16([2.0 ** -17, 2.0 ** -18], [1.0, 1.0]) == 2.0 ** -16  # subnormal quantum 2^-17: 1.5 quanta ties to 2
+    # one rounding per step, of the fused multiply-add
+    assert chain16([3.0, 1.0 + 2.0 ** -11], [1.0 / 3.0, 3.0]) == float(
+        L.lamp_oracle_rne_e4m11(float(np.float64(np.float32(1.0 + 2.0 ** -11)) * 3.0
+                                      + np.float64(L.lamp_oracle_rne_e4m11(float(np.float32(3.0) * np.float32(1.0 / 3.0)))))))
+
+
+def test_per_step_mode_agrees_when_partial_sums_are_representable(small):
+    """Small-integer inputs with a power-of-two scale: every partial sum is exact in 12 bits, so the per-step
+    recursion and the single-rounding reading give the same 16-bit logits and therefore the same outputs;
+    on the Qwen-shaped inputs they differ, and the per-step one is the less accurate."""
+    g = torch.Generator().manual_seed(5)
+    q = torch.randint(-3, 4, (1, 2, 256, 128), generator=g).to(torch.bfloat16)
+    k = torch.randint(-3, 4, (1, 1, 256, 128), generator=g).to(torch.bfloat16)
+    v = torch.randn(1, 1, 256, 128, generator=g).to(torch.bfloat16)
+    a = oracle.run_all(q, k, v, scale=2.0 ** -4, flags=oracle.FORCE_16BIT)
+    b = oracle.run_all(q, k, v, scale=2.0 ** -4, flags=oracle.FORCE_16BIT | oracle.H16_SEQ)
+    assert np.array_equal(a.out, b.out) and np.array_equal(a.lse, b.lse)
+    qq, kk, vv, sc = small
+    a = oracle.run_all(qq, kk, vv, scale=sc, flags=oracle.FORCE_16BIT)
+    b = oracle.run_all(qq, kk, vv, scale=sc, flags=oracle.FORCE_16BIT | oracle.H16_SEQ)
+    o, _, _ = ref_attention(qq, kk, vv, sc)
+    ea = (dense(a, 1, 4, 512, 128)[0] - o).norm(); eb = (dense(b, 1, 4, 512, 128)[0] - o).norm()
+    assert not np.array_equal(a.out, b.out) and ea < eb < 50 * ea
+
+
 def test_overflow_rule_of_section_3_3():
     f = GOLD["logit_bound_factor"]
     assert abs(f - 8 * math.sqrt(2)) < 1e-12
