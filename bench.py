@@ -7,7 +7,7 @@ input (B=4, 32 query / 8 KV heads, N=8192, head_dim 128, causal).  Prints ONE JS
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config C]
                   [--mode lamp|force8|force16] [--tau T] [--delta D] [--no-stage1]
-                  [--compact] [--scale-mult M] [--window W]
+                  [--compact] [--h16-seq] [--scale-mult M] [--window W]
 
 The options after --config select the other workloads and the paper's ablations (threshold
 and margin sweeps, stage 1 off, the scale sweep of the long-context config, the sliding
@@ -139,7 +139,7 @@ def oracle_sample_run(cfg, q, k, v, scale, n_units, seed=11, knobs=None):
 
 def knobs_of(args):
     """Thresholds, mode bits and mask of this run (the same numeric flag values in the library and the oracle)."""
-    flags = {"lamp": 0, "force8": 2, "force16": 1}[args.mode] | (4 if args.no_stage1 else 0) | (16 if args.compact else 0)
+    flags = {"lamp": 0, "force8": 2, "force16": 1}[args.mode] | (4 if args.no_stage1 else 0) | (16 if args.compact else 0) | (32 if args.h16_seq else 0)
     return {"tau": args.tau, "delta": args.delta, "flags": flags, "window": args.window}
 
 
@@ -184,6 +184,8 @@ def workload_config(cfg, args):
         extra += ", stage 1 off"
     if args.compact:
         extra += ", compact-layout branch"
+    if args.h16_seq:
+        extra += ", per-step e4m11 accumulation"
     return {"workload": f"config {cfg.index}: {cfg.name} prefill, B={cfg.B}, Hq={cfg.Hq}, Hkv={cfg.Hkv}, "
                         f"N={cfg.N}, head_dim={cfg.D}, causal{extra}, tau={args.tau:g}, delta=2^{math.log2(args.delta):g}",
             "l2": "inputs (Q+K+V+O = %.0f MB) larger than the 126 MB L2" %
@@ -205,6 +207,8 @@ def main():
     ap.add_argument("--no-stage1", action="store_true", help="the ablation without the running-maximum test")
     ap.add_argument("--compact", action="store_true",
                     help="the compact register layout's branch: two or more marked sub-blocks send the tile to 16 bits")
+    ap.add_argument("--h16-seq", action="store_true",
+                    help="16-bit logits by per-step e4m11 accumulation (the other reading of the 16-bit accumulate)")
     ap.add_argument("--scale-mult", type=float, default=1.0, help="softmax scale = mult / sqrt(head_dim)")
     ap.add_argument("--window", type=int, default=0, help="sliding window (0 = global causal)")
     args = ap.parse_args()
@@ -308,7 +312,7 @@ def main():
     peak = 4.0 / MIN_SLOTS_PER_STEP * SM_COUNT * LANES_PER_SM * SM_MAX_MHZ * 1e6 / 1e12
     # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu capture summarised in
     # profiles/lamp_fwd_sm100_config2_ncu_full.txt (algorithmic bytes: 680 MB)
-    headline = (args.mode == "lamp" and not args.no_stage1 and not args.compact and args.tau == 0.5 and args.delta == 2.0 ** -8
+    headline = (args.mode == "lamp" and not args.no_stage1 and not args.compact and not args.h16_seq and args.tau == 0.5 and args.delta == 2.0 ** -8
                 and args.scale_mult == 1.0 and args.window == 0)
     traffic = {2: 655.97e6}.get(cfg.index) if headline else None
     roofline = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",

@@ -54,6 +54,11 @@ typedef enum lamp_attn_error {
  * (batch, head, token); the head_dim stride is 1.  Every row start must be
  * 16-byte aligned (strides multiples of 8 elements, base pointers 16-byte
  * aligned). */
+#define LAMP_H16_SEQ         0x20u /* 16-bit logits by the recursion of Sec. 4.1, c <- round_e4m11(c + k q) on
+                                      the pre-scaled query, every partial sum rounded, instead of the exact dot
+                                      product rounded once (the library's default reading of the 16-bit
+                                      accumulation); much slower on this GPU, for comparison only          */
+
 typedef struct lamp_attn_params {
   int32_t batch, heads_q, heads_kv; /* heads_q % heads_kv == 0 (grouped-query attention)      */
   int32_t seqlen;                   /* multiple of 128                                         */

@@ -7,7 +7,7 @@ import os
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "liblamp_attn.so")
 
-LAMP_FORCE_16BIT, LAMP_FORCE_8BIT, LAMP_NO_STAGE1, LAMP_OUT_FP32, LAMP_COMPACT_BRANCH = 1, 2, 4, 8, 16
+LAMP_FORCE_16BIT, LAMP_FORCE_8BIT, LAMP_NO_STAGE1, LAMP_OUT_FP32, LAMP_COMPACT_BRANCH, LAMP_H16_SEQ = 1, 2, 4, 8, 16, 32
 
 EXPORTS = ("lamp_attn_default_params", "lamp_attn_contiguous_strides", "lamp_attn_workspace_bytes",
            "lamp_attn_fwd", "lamp_attn_fwd_digest", "lamp_attn_debug_round_e4m3", "lamp_attn_get_stats", "lamp_attn_last_cuda_error", "lamp_attn_strerror")

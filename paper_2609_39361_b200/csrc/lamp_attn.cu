@@ -163,7 +163,7 @@ static int check_params(const void* q, const void* k, const void* v, void* out,
   if (p->heads_q % p->heads_kv) return LAMP_ERR_INVALID_ARG;
   if (!(p->threshold >= 0.0f) || !(p->delta >= 0.0f) || !isfinite(p->scale)) return LAMP_ERR_INVALID_ARG;
   if (p->window < 0 || (p->window > 0 && !p->causal)) return LAMP_ERR_INVALID_ARG;
-  if (p->flags & ~(LAMP_FORCE_16BIT | LAMP_FORCE_8BIT | LAMP_NO_STAGE1 | LAMP_OUT_FP32 | LAMP_COMPACT_BRANCH))
+  if (p->flags & ~(LAMP_FORCE_16BIT | LAMP_FORCE_8BIT | LAMP_NO_STAGE1 | LAMP_OUT_FP32 | LAMP_COMPACT_BRANCH | LAMP_H16_SEQ))
     return LAMP_ERR_INVALID_ARG;
   if ((p->flags & LAMP_FORCE_16BIT) && (p->flags & (LAMP_FORCE_8BIT | LAMP_NO_STAGE1)))
     return LAMP_ERR_INVALID_ARG;

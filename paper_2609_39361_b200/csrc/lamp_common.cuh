@@ -74,6 +74,15 @@ __device__ __forceinline__ float rne_e4m11(double x) {
   return copysignf((float)r, (float)x);
 }
 
+// The same rounding of an fp32 value (the per-step 16-bit accumulation mode).
+__device__ __forceinline__ float rne_e4m11_f(float t) {
+  const float a = fabsf(t);
+  float r;
+  if (a < 0.015625f) r = __fsub_rn(__fadd_rn(a, 96.0f), 96.0f);   // multiples of 2^-17: the ulp of [64, 128)
+  else r = fminf(rne_sig12(a), 448.0f);
+  return copysignf(r, t);
+}
+
 // 16-bit exponential: exp(a) correctly rounded to 12 significant bits, with the
 // subnormal quantum 2^-41 below 2^-30 (ue5m11 with the bias that maps 0xF800 to 1.0).
 __device__ __forceinline__ float exp16(float a) {

@@ -225,6 +225,64 @@ __device__ __noinline__ void dot16(const __nv_bfloat16* __restrict__ krow, int64
   ptx::tmem_wait_st();
 }
 
+// The same 16 x 32 logits by the other reading of the 16-bit accumulation (mode LAMP_H16_SEQ): the
+// recursion of the first pass, c <- RNE_e4m11(fma(k, q*scale, c)), every partial sum rounded.  Plain
+// fp32 work on the lane's 4 queries x 4 keys; a comparison mode, not tuned.
+// q_quad: the lane's quad in the shared-memory Q operand of the chain (fp32 q*scale for head_dim 128,
+// raw bf16 q for 256); K rows from global memory, 16 bytes (8 channels) per key at a time.
+template <int D>
+__device__ __noinline__ void dot16_seq(const __nv_bfloat16* __restrict__ krow, int64_t kstride,
+                                       const unsigned char* q_quad, float scale, uint32_t tdst) {
+  constexpr bool QF32 = (D == 128);
+  const int tp = threadIdx.x & 3;
+  float acc[4][4];
+#pragma unroll
+  for (int a = 0; a < 4; ++a)
+#pragma unroll
+    for (int b = 0; b < 4; ++b) acc[a][b] = 0.0f;
+  const __nv_bfloat16* ksrc = krow + (int64_t)(4 * tp) * kstride;
+  uint4 kraw[4];
+#pragma unroll
+  for (int b = 0; b < 4; ++b) kraw[b] = *reinterpret_cast<const uint4*>(ksrc + b * kstride);
+#pragma unroll 1
+  for (int k0 = 0; k0 < D; k0 += 8) {
+    uint4 cur[4];
+#pragma unroll
+    for (int b = 0; b < 4; ++b) cur[b] = kraw[b];
+    const int kn = (k0 + 8) & (D - 1);
+#pragma unroll
+    for (int b = 0; b < 4; ++b) kraw[b] = *reinterpret_cast<const uint4*>(ksrc + b * kstride + kn);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      float q4[4];
+      if (QF32) {
+        const float4 qv = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(q_quad) + (k0 + e) * kBM);
+        q4[0] = qv.x; q4[1] = qv.y; q4[2] = qv.z; q4[3] = qv.w;
+      } else {
+        const uint2 qh = *reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(q_quad) + (k0 + e) * kBM);
+        q4[0] = __fmul_rn(__uint_as_float(qh.x << 16), scale);
+        q4[1] = __fmul_rn(__uint_as_float(qh.x & 0xffff0000u), scale);
+        q4[2] = __fmul_rn(__uint_as_float(qh.y << 16), scale);
+        q4[3] = __fmul_rn(__uint_as_float(qh.y & 0xffff0000u), scale);
+      }
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        const uint32_t w = (&cur[b].x)[e >> 1];
+        const float kv = __uint_as_float((e & 1) ? (w & 0xffff0000u) : (w << 16));
+#pragma unroll
+        for (int a = 0; a < 4; ++a) acc[a][b] = rne_e4m11_f(__fmaf_rn(kv, q4[a], acc[a][b]));
+      }
+    }
+  }
+  uint32_t yr[16];
+#pragma unroll
+  for (int a = 0; a < 4; ++a)
+#pragma unroll
+    for (int b = 0; b < 4; ++b) yr[4 * a + b] = __float_as_uint(acc[a][b]);
+  ptx::tmem_st16(tdst, yr);
+  ptx::tmem_wait_st();
+}
+
 // active, s1, s2, hist, bigrow are warp-uniform; sat8, sat16, gt1 are per-lane partial counts.
 struct WarpCounters {
   unsigned long long active, s1, s2, hist[5], bigrow;
@@ -281,13 +339,18 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
                                               uint32_t tscratch, uint32_t& lo_dirty, RowState& st,
                                               float (&lam)[4], WarpCounters& wc, unsigned long long (&cks)[2],
                                               int dump_row0, int row0, long long* ph, uint64_t* pv_bar,
-                                              uint32_t pv_parity, bool pv_wait, int* status, bool& ok) {
+                                              uint32_t pv_parity, bool pv_wait, int* status, bool& ok, const unsigned char* q_quad) {
   const int lane = threadIdx.x & 31;
   const int qa = lane >> 2, th_own = lane & 3;
   const double scale_d = (double)P.scale;
   const bool force16 = P.flags & LAMP_FORCE_16BIT;
   const bool force8 = P.flags & LAMP_FORCE_8BIT;
   const bool skip1 = (P.flags & (LAMP_FORCE_8BIT | LAMP_NO_STAGE1)) != 0;
+  auto logits16 = [&](int th) {
+    const __nv_bfloat16* kr = ktile + (int64_t)(16 * th) * kstride;
+    if (P.flags & LAMP_H16_SEQ) dot16_seq<D>(kr, kstride, q_quad, P.scale, tscratch + 16 * th);
+    else dot16<D>(kr, kstride, tq, dscr, scale_d, tscratch + 16 * th);
+  };
 
   // ---- per sub-block, per query maxima; which sub-blocks are active --------------------------
   // yw[4a + c] packs the first-pass logits of query a, keys 4c..4c+3 of the lane's sub-block
@@ -365,7 +428,7 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
     if (!fail) continue;
     Theta |= 1u << th;
     LAMP_TIC(t_d1);
-    dot16<D>(ktile + (int64_t)(16 * th) * kstride, kstride, tq, dscr, scale_d, tscratch + 16 * th);   // results parked in TMEM
+    logits16(th);   // results parked in TMEM
     LAMP_TOC(4, t_d1);
     uint32_t yr[16];
     ptx::tmem_ld16(tscratch + 16 * th, yr);
@@ -640,7 +703,7 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
   for (int th = 0; th < 4; ++th) {
     if (!((Rset >> th) & 1u)) continue;
     LAMP_TIC(t_d2);
-    dot16<D>(ktile + (int64_t)(16 * th) * kstride, kstride, tq, dscr, scale_d, tscratch + 16 * th);
+    logits16(th);
     LAMP_TOC(4, t_d2);
     uint32_t yr[16];
     ptx::tmem_ld16(tscratch + 16 * th, yr);
@@ -953,6 +1016,7 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
     const bool dump_rows = DUMP && b == P.dbg_batch && h == P.dbg_head;
     const __nv_bfloat16* kg = P.k + b * P.ks[0] + hk * P.ks[1];
     double* dscr = dscr_all + grp * 384;
+    const unsigned char* q_quad = qs + (QF32 ? 4 : 2) * (grp * kBQ + 4 * qa);
     const uint32_t tlane = tbase + ((uint32_t)(grp * 32) << 16);
     const uint32_t tscr = tlane + kColScr, tq = tlane + kColQ, tring = tlane + kColRing;
     {
@@ -1020,11 +1084,11 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
         if (full)
           flag = lamp_post<D, true, DUMP>(P, g, yw, ktile, P.ks[2], tq, lut, dscr, phi, plo, tscr, lo_dirty,
                                           st, lam, wc, cks, dump0, grp * kBQ, ph, &bars[kPvDone0 + grp], (n - 1) & 1, n > 0,
-                                          status, ok);
+                                          status, ok, q_quad);
         else
           flag = lamp_post<D, false, DUMP>(P, g, yw, ktile, P.ks[2], tq, lut, dscr, phi, plo, tscr, lo_dirty,
                                            st, lam, wc, cks, dump0, grp * kBQ, ph, &bars[kPvDone0 + grp], (n - 1) & 1, n > 0,
-                                           status, ok);
+                                           status, ok, q_quad);
       } else {
         // no visible pair for this group: its rows of the P tile are zero (once the previous
         // P V product has read them)

@@ -78,11 +78,14 @@ def test_scale_sweep_saturation(mult):
                                              (oracle.NO_STAGE1, 0.25, 2.0 ** -4), (0, 0.0, 2.0 ** -8),
                                              (oracle.COMPACT_BRANCH, 0.5, 2.0 ** -8),
                                              (oracle.COMPACT_BRANCH, 0.125, 2.0 ** -8),
-                                             (oracle.COMPACT_BRANCH | oracle.NO_STAGE1, 0.125, 2.0 ** -8)])
+                                             (oracle.COMPACT_BRANCH | oracle.NO_STAGE1, 0.125, 2.0 ** -8),
+                                             (oracle.H16_SEQ, 0.5, 2.0 ** -8), (oracle.H16_SEQ, 0.125, 2.0 ** -8),
+                                             (oracle.H16_SEQ | oracle.FORCE_16BIT, 0.5, 2.0 ** -8)])
 def test_threshold_and_margin_sweeps(flags, tau, delta):
     """Points of the ablation sweeps (threshold of eq. (8), margin of eq. (7), stage 1 off): where
     stage 2 does most of the flagging, and tau = 0, which recomputes whatever carries any mass; the
-    branch of the compact register layout (Sec. 3.3) on top of them."""
+    branch of the compact register layout (Sec. 3.3) and the per-step reading of the 16-bit accumulation
+    (Sec. 4.1) on top of them."""
     cfg = li.CONFIGS[1]
     q, k, v = li.make_qkv(cfg, Hq=4, Hkv=2, N=512, seed=31)
     sc = li.softmax_scale(cfg.D)
@@ -92,7 +95,7 @@ def test_threshold_and_margin_sweeps(flags, tau, delta):
     compare_dense_bytes(gpu, ref, 0, 1)
 
 
-@pytest.mark.parametrize("window,flags", [(0, 0), (192, 0), (0, oracle.FORCE_16BIT)])
+@pytest.mark.parametrize("window,flags", [(0, 0), (192, 0), (0, oracle.FORCE_16BIT), (0, oracle.H16_SEQ)])
 def test_head_dim_256_gemma_shaped(window, flags):
     """head_dim 256 (two 128-channel halves per tile), global and sliding-window layers."""
     cfg = li.CONFIGS[3]
