@@ -94,9 +94,12 @@ static int ensure_device(int* dev_out) {
     if (!fn || qr != cudaDriverEntryPointSuccess) return cuda_fail(cudaErrorNotSupported);
     g_encode = (TensorMapEncodeFn)fn;
   }
-  const void* kernels[4] = {(const void*)lamp_fwd_sm100<128, false>, (const void*)lamp_fwd_sm100<128, true>,
-                            (const void*)lamp_fwd_sm100<256, false>, (const void*)lamp_fwd_sm100<256, true>};
-  for (int i = 0; i < 4; ++i) {
+  const void* kernels[8] = {
+      (const void*)lamp_fwd_sm100<128, false, false>, (const void*)lamp_fwd_sm100<128, true, false>,
+      (const void*)lamp_fwd_sm100<256, false, false>, (const void*)lamp_fwd_sm100<256, true, false>,
+      (const void*)lamp_fwd_sm100<128, false, true>,  (const void*)lamp_fwd_sm100<128, true, true>,
+      (const void*)lamp_fwd_sm100<256, false, true>,  (const void*)lamp_fwd_sm100<256, true, true>};
+  for (int i = 0; i < 8; ++i) {
     e = cudaFuncSetAttribute(kernels[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLaunch);
     if (e != cudaSuccess) return cuda_fail(e);
   }
@@ -233,13 +236,17 @@ int lamp_attn_fwd(const void* q, const void* k, const void* v, void* out, float*
   dim3 grid(p->seqlen / kBM, p->heads_q, p->batch), block(kThreads);
   const uint2* lutp = (const uint2*)lut_ptr;
   DeviceStats* dsp = (DeviceStats*)stats_ptr;
+#define LAMP_LAUNCH(D_, DUMP_, SEQ_) \
+  lamp_fwd_sm100<D_, DUMP_, SEQ_><<<grid, block, kSmemLaunch, stream>>>(P, kmap, vmap, lutp, dsp)
+  const bool seq16 = (p->flags & LAMP_H16_SEQ) != 0;   // the per-step 16-bit accumulation has kernels of its own
   if (p->head_dim == 128) {
-    if (dump) lamp_fwd_sm100<128, true><<<grid, block, kSmemLaunch, stream>>>(P, kmap, vmap, lutp, dsp);
-    else lamp_fwd_sm100<128, false><<<grid, block, kSmemLaunch, stream>>>(P, kmap, vmap, lutp, dsp);
+    if (seq16) { if (dump) LAMP_LAUNCH(128, true, true); else LAMP_LAUNCH(128, false, true); }
+    else       { if (dump) LAMP_LAUNCH(128, true, false); else LAMP_LAUNCH(128, false, false); }
   } else {
-    if (dump) lamp_fwd_sm100<256, true><<<grid, block, kSmemLaunch, stream>>>(P, kmap, vmap, lutp, dsp);
-    else lamp_fwd_sm100<256, false><<<grid, block, kSmemLaunch, stream>>>(P, kmap, vmap, lutp, dsp);
+    if (seq16) { if (dump) LAMP_LAUNCH(256, true, true); else LAMP_LAUNCH(256, false, true); }
+    else       { if (dump) LAMP_LAUNCH(256, true, false); else LAMP_LAUNCH(256, false, false); }
   }
+#undef LAMP_LAUNCH
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
   return LAMP_OK;

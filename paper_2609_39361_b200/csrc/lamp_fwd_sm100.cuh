@@ -332,7 +332,7 @@ __device__ __forceinline__ uint32_t enc_exp8(float e) {
 // The 64 first-pass logits of a lane arrive packed in 16 words (yw) and are unpacked 16 at a
 // time, so that the per-element work is a short loop instead of a long unrolled stretch of
 // code and the registers are free for the 16-bit path.
-template <int D, bool FULL, bool DUMP>
+template <int D, bool FULL, bool DUMP, bool SEQ16>
 __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileGeom& g, const uint32_t (&yw)[16],
                                               const __nv_bfloat16* ktile, int64_t kstride, uint32_t tq,
                                               const uint2* lut, double* dscr, unsigned char* phi, unsigned char* plo,
@@ -348,7 +348,7 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
   const bool skip1 = (P.flags & (LAMP_FORCE_8BIT | LAMP_NO_STAGE1)) != 0;
   auto logits16 = [&](int th) {
     const __nv_bfloat16* kr = ktile + (int64_t)(16 * th) * kstride;
-    if (P.flags & LAMP_H16_SEQ) dot16_seq<D>(kr, kstride, q_quad, P.scale, tscratch + 16 * th);
+    if constexpr (SEQ16) dot16_seq<D>(kr, kstride, q_quad, P.scale, tscratch + 16 * th);
     else dot16<D>(kr, kstride, tq, dscr, scale_d, tscratch + 16 * th);
   };
 
@@ -760,7 +760,9 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
 }
 
 
-template <int D, bool DUMP>
+// SEQ16: the per-step reading of the 16-bit accumulation (mode LAMP_H16_SEQ), a kernel of its own so that
+// the default one carries nothing of it (code that never ran still cost it 2.5 % through register allocation).
+template <int D, bool DUMP, bool SEQ16>
 __global__ void __launch_bounds__(kThreads, 1)
 lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ CUtensorMap kmap,
                const __grid_constant__ CUtensorMap vmap, const uint2* __restrict__ lut_g,
@@ -1016,7 +1018,7 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
     const bool dump_rows = DUMP && b == P.dbg_batch && h == P.dbg_head;
     const __nv_bfloat16* kg = P.k + b * P.ks[0] + hk * P.ks[1];
     double* dscr = dscr_all + grp * 384;
-    const unsigned char* q_quad = qs + (QF32 ? 4 : 2) * (grp * kBQ + 4 * qa);
+    const unsigned char* q_quad = SEQ16 ? qs + (QF32 ? 4 : 2) * (grp * kBQ + 4 * qa) : nullptr;
     const uint32_t tlane = tbase + ((uint32_t)(grp * 32) << 16);
     const uint32_t tscr = tlane + kColScr, tq = tlane + kColQ, tring = tlane + kColRing;
     {
@@ -1082,11 +1084,11 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
         const int dump0 = dump_rows ? j0 : -1;
         const __nv_bfloat16* ktile = kg + (int64_t)i0 * P.ks[2];
         if (full)
-          flag = lamp_post<D, true, DUMP>(P, g, yw, ktile, P.ks[2], tq, lut, dscr, phi, plo, tscr, lo_dirty,
+          flag = lamp_post<D, true, DUMP, SEQ16>(P, g, yw, ktile, P.ks[2], tq, lut, dscr, phi, plo, tscr, lo_dirty,
                                           st, lam, wc, cks, dump0, grp * kBQ, ph, &bars[kPvDone0 + grp], (n - 1) & 1, n > 0,
                                           status, ok, q_quad);
         else
-          flag = lamp_post<D, false, DUMP>(P, g, yw, ktile, P.ks[2], tq, lut, dscr, phi, plo, tscr, lo_dirty,
+          flag = lamp_post<D, false, DUMP, SEQ16>(P, g, yw, ktile, P.ks[2], tq, lut, dscr, phi, plo, tscr, lo_dirty,
                                            st, lam, wc, cks, dump0, grp * kBQ, ph, &bars[kPvDone0 + grp], (n - 1) & 1, n > 0,
                                            status, ok, q_quad);
       } else {
