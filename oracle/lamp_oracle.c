@@ -45,6 +45,8 @@
 #define LAMP_FORCE_8BIT  2u
 #define LAMP_NO_STAGE1   4u
 #define LAMP_COMPACT_BRANCH 16u  /* Sec. 3.3 "Register layout": the compact layout's branch (see below) */
+#define LAMP_SR_E4M3     64u     /* stochastic rounding in the 8-bit accumulation (Sec. 3.3, last sentence of the
+                                    paragraph on formats), see lamp_oracle_sr_e4m3 */
 #define LAMP_H16_SEQ     32u     /* 16-bit logits by per-step e4m11 accumulation (the other reading, see logit16) */
 
 typedef struct {
@@ -52,6 +54,7 @@ typedef struct {
   int32_t causal, window;
   float scale, tau, delta;
   uint32_t flags;
+  uint32_t sr_seed;      /* seed of the counter-based generator of LAMP_SR_E4M3 */
 } lamp_oracle_params;
 
 typedef struct {
@@ -205,6 +208,8 @@ uint32_t lamp_oracle_stage2(const double xi[NK][BQ], const float* omega_hat, flo
 }
 
 float lamp_oracle_chain16(const float* a, const float* b, int n);
+float lamp_oracle_sr_e4m3(float t, uint32_t u20);
+uint32_t lamp_oracle_sr_bits(uint32_t seed, uint32_t bh, uint32_t j, uint32_t i, uint32_t kk);
 
 /* A 16-bit logit (Alg. 1 "recompute Y_theta in high precision").
  * Default reading: the exact dot product as a sequential fp64 fma chain over the channels, times the
@@ -309,7 +314,14 @@ static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
       for (int j = 0; j < BQ; ++j) {
         float c = 0.0f;
         for (int kk = 0; kk < D; ++kk)
-          c = lamp_oracle_rne_e4m3(fmaf(bf16_to_float(K[(i0 + i) * D + kk]), qs[j * D + kk], c));
+          {
+            float tkk = fmaf(bf16_to_float(K[(i0 + i) * D + kk]), qs[j * D + kk], c);
+            if (p->flags & LAMP_SR_E4M3)
+              c = lamp_oracle_sr_e4m3(tkk, lamp_oracle_sr_bits(p->sr_seed, (uint32_t)(b * p->heads_q + h),
+                                                               (uint32_t)(j0 + j), (uint32_t)(i0 + i), (uint32_t)kk));
+            else
+              c = lamp_oracle_rne_e4m3(tkk);
+          }
         Y8[i][j] = c;
       }
 
@@ -530,6 +542,38 @@ int lamp_oracle_units(const uint16_t* q, const uint16_t* k, const uint16_t* v,
 void lamp_oracle_rne_e4m3_array(const float* in, float* out, int64_t n) {
 #pragma omp parallel for schedule(static)
   for (int64_t i = 0; i < n; ++i) out[i] = lamp_oracle_rne_e4m3(in[i]);
+}
+
+/* Stochastic rounding onto the e4m3 grid (Sec. 3.3 proposes it against swamping; the paper does not
+ * specify it further).  Reading taken here, in integer arithmetic so that any two implementations agree
+ * bit for bit: with u a uniform 20-bit integer, the magnitude's fp32 bit pattern plus u, with the 20
+ * mantissa bits below e4m3's three cleared, is the result: the value goes up to the next grid point
+ * with probability (distance from the lower one) / (spacing), exactly, in units of 2^-20.  Below 2^-6
+ * (the subnormal range, fixed spacing 2^-9) the magnitude is first moved into [2^-6, 2^-5), whose
+ * spacing is 2^-9, by one fp32 addition, and moved back afterwards.  Magnitudes beyond 448 saturate. */
+float lamp_oracle_sr_e4m3(float t, uint32_t u20) {
+  float a = fabsf(t);
+  float off = a < 0.015625f ? 0.015625f : 0.0f;
+  float s = a + off;
+  uint32_t bits;
+  memcpy(&bits, &s, 4);
+  bits = (bits + (u20 & 0xFFFFFu)) & 0xFFF00000u;
+  float r;
+  memcpy(&r, &bits, 4);
+  r = r - off;
+  if (r > 448.0f) r = 448.0f;
+  return copysignf(r, t);
+}
+
+/* The 20 random bits of one accumulation step: a counter-based generator (a 32-bit integer hash of
+ * the step's coordinates: batch * heads + head, absolute query row, absolute key, channel), so that
+ * every implementation draws the same bits whatever its order of evaluation. */
+uint32_t lamp_oracle_sr_bits(uint32_t seed, uint32_t bh, uint32_t j, uint32_t i, uint32_t kk) {
+  uint32_t x = seed ^ (bh * 0x27D4EB2Fu) ^ (j * 0x85EBCA77u) ^ (i * 0x9E3779B1u) ^ (kk * 0xC2B2AE3Du);
+  x ^= x >> 16; x *= 0x7FEB352Du;
+  x ^= x >> 15; x *= 0x846CA68Bu;
+  x ^= x >> 16;
+  return x >> 12;
 }
 
 /* The same recursion on the 16-bit grid: c <- RNE_e4m11(fmaf(a[t], b[t], c)), t ascending, c0 = +0

@@ -18,6 +18,7 @@ _SRC = os.path.join(_HERE, "lamp_oracle.c")
 _SO = os.path.join(_HERE, "liblamp_oracle.so")
 
 FORCE_16BIT, FORCE_8BIT, NO_STAGE1 = 1, 2, 4
+SR_E4M3 = 64          # stochastic rounding in the 8-bit accumulation (Sec. 3.3), counter-based generator
 H16_SEQ = 32          # 16-bit logits by per-step e4m11 accumulation (Sec. 4.1 recursion) instead of one rounding
 COMPACT_BRANCH = 16   # Sec. 3.3 'Register layout': whole tile to 16 bits once two sub-blocks are marked
 
@@ -26,7 +27,7 @@ class Params(C.Structure):
     _fields_ = [("batch", C.c_int32), ("heads_q", C.c_int32), ("heads_kv", C.c_int32),
                 ("seqlen", C.c_int32), ("head_dim", C.c_int32), ("causal", C.c_int32),
                 ("window", C.c_int32), ("scale", C.c_float), ("tau", C.c_float),
-                ("delta", C.c_float), ("flags", C.c_uint32)]
+                ("delta", C.c_float), ("flags", C.c_uint32), ("sr_seed", C.c_uint32)]
 
 
 class Stats(C.Structure):
@@ -70,6 +71,10 @@ def lib():
         L.lamp_oracle_exp16.restype = f32; L.lamp_oracle_exp16.argtypes = [f32]
         L.lamp_oracle_stage2.restype = u32
         L.lamp_oracle_stage2.argtypes = [C.c_void_p, C.c_void_p, f32, u32]
+        L.lamp_oracle_sr_e4m3.restype = f32
+        L.lamp_oracle_sr_e4m3.argtypes = [f32, C.c_uint32]
+        L.lamp_oracle_sr_bits.restype = C.c_uint32
+        L.lamp_oracle_sr_bits.argtypes = [C.c_uint32] * 5
         L.lamp_oracle_chain16.restype = f32
         L.lamp_oracle_chain16.argtypes = [C.c_void_p, C.c_void_p, C.c_int]
         L.lamp_oracle_chain8.restype = f32
@@ -113,7 +118,7 @@ def _bits(x) -> np.ndarray:
 
 
 def run_units(q, k, v, units, *, causal=True, window=0, scale=None, tau=0.5, delta=2.0 ** -8,
-              flags=0, dumps=False, checksums=True) -> OracleResult:
+              flags=0, sr_seed=0, dumps=False, checksums=True) -> OracleResult:
     """Run the oracle on the listed (b, h, g) units.  q: [B, Hq, N, D], k/v: [B, Hkv, N, D]."""
     qb, kb, vb = _bits(q), _bits(k), _bits(v)
     B, Hq, N, D = qb.shape
@@ -122,7 +127,7 @@ def run_units(q, k, v, units, *, causal=True, window=0, scale=None, tau=0.5, del
         scale = np.float32(1.0 / np.sqrt(float(D)))
     units = np.ascontiguousarray(np.asarray(units, dtype=np.int32).reshape(-1, 3))
     n = units.shape[0]
-    p = Params(B, Hq, Hkv, N, D, int(causal), int(window), float(scale), float(tau), float(delta), int(flags))
+    p = Params(B, Hq, Hkv, N, D, int(causal), int(window), float(scale), float(tau), float(delta), int(flags), int(sr_seed))
     out = np.zeros((n, 32, D), np.float32)
     lse = np.zeros((n, 32), np.float32)
     fl = np.zeros((n, N // 64), np.uint8)

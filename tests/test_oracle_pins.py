@@ -142,6 +142,68 @@ def test_per_step_mode_agrees_when_partial_sums_are_representable(small):
     assert not np.array_equal(a.out, b.out) and ea < eb < 50 * ea
 
 
+def test_stochastic_rounding_is_exactly_proportional():
+    """Stochastic rounding of the 8-bit accumulation (Sec. 3.3): the result is one of the two grid neighbours,
+    grid values never move, and over all 2^20 random integers the number of round-ups is exactly the
+    distance to the lower neighbour in units of spacing / 2^20 - so the mean is the value itself."""
+    sr = L.lamp_oracle_sr_e4m3
+    grid = sorted(g for g in E4M3_GRID if g >= 0)
+    for g in grid[::7] + [448.0]:
+        for u in (0, 1, 0x7FFFF, 0xFFFFF):
+            assert sr(g, u) == g and sr(-g, u) == -g
+    #  value, lower neighbour, upper neighbour, round-ups out of 2^20 (worked by hand)
+    cases = [(1.0 + 2.0 ** -5, 1.0, 1.125, 1 << 18),                 # a quarter of the way up
+             (-(2.5 + 3 * 2.0 ** -4), -2.5, -2.75, 3 << 18),           # negative: away from zero with p = 3/4
+             (300.0, 288.0, 320.0, (12 << 20) // 32),                 # spacing 32 at 2^8
+             (2.0 ** -9 * 2.25, 2.0 ** -8, 3 * 2.0 ** -9, 1 << 18),     # subnormal range, spacing 2^-9
+             (2.0 ** -6 - 2.0 ** -11, 7 * 2.0 ** -9, 2.0 ** -6, 3 << 18),  # top of the subnormal range
+             (2.0 ** -12, 0.0, 2.0 ** -9, 1 << 17)]
+    for t, lo, hi, ups in cases:
+        step = 64
+        got = [sr(t, u) for u in range(0, 1 << 20, step)]
+        assert set(got) <= {lo, hi}, (t, set(got))
+        assert sum(x == hi for x in got) * step == ups, t
+        assert sr(t, 0) == lo and sr(t, 0xFFFFF) == (hi if ups else lo)
+    assert sr(470.0, 0) == 448.0 and sr(470.0, 0xFFFFF) == 448.0 and sr(-1e6, 5) == -448.0
+    assert sr(447.0, 0xFFFFF) == 448.0 and sr(447.0, 0) == 416.0
+
+
+def test_stochastic_rounding_lifts_the_swamped_chain():
+    """The swamping example of the accumulation pins: 128 ones stall at 16 under round-to-nearest; with
+    stochastic rounding the chain is unbiased, its mean over seeds is the true sum 128."""
+    sr, bits = L.lamp_oracle_sr_e4m3, L.lamp_oracle_sr_bits
+    tot = []
+    for seed in range(400):
+        c = 0.0
+        for kk in range(128):
+            c = sr(float(np.float32(c) + np.float32(1.0)), bits(seed, 3, 17, 5, kk))
+        tot.append(c)
+    tot = np.array(tot)
+    assert abs(tot.mean() - 128.0) < 4.0 and tot.std() > 8.0
+    # the generator: 20 bits, reproducible, sensitive to every coordinate, uniform
+    u = np.array([bits(1, 0, j, i, kk) for j in range(8) for i in range(50) for kk in range(50)])
+    assert u.max() < (1 << 20) and abs(u.mean() / (1 << 20) - 0.5) < 0.01
+    assert abs(np.mean((u >> 19) & 1) - 0.5) < 0.02 and abs(np.mean(u & 1) - 0.5) < 0.02
+    base = bits(7, 1, 2, 3, 4)
+    assert base == bits(7, 1, 2, 3, 4)
+    assert len({base, bits(8, 1, 2, 3, 4), bits(7, 2, 2, 3, 4), bits(7, 1, 3, 3, 4), bits(7, 1, 2, 4, 4),
+                bits(7, 1, 2, 3, 5)}) == 6
+
+
+def test_stochastic_rounding_end_to_end_is_seeded_and_consistent(small):
+    q, k, v, sc = small
+    a = oracle.run_all(q, k, v, scale=sc, flags=oracle.SR_E4M3, sr_seed=11, dumps=True)
+    b = oracle.run_all(q, k, v, scale=sc, flags=oracle.SR_E4M3, sr_seed=11, dumps=True)
+    c = oracle.run_all(q, k, v, scale=sc, flags=oracle.SR_E4M3, sr_seed=12, dumps=True)
+    r = oracle.run_all(q, k, v, scale=sc, dumps=True)
+    assert np.array_equal(a.y8, b.y8) and np.array_equal(a.out, b.out)
+    assert not np.array_equal(a.y8, c.y8) and not np.array_equal(a.y8, r.y8)
+    # first-pass logits stay on the e4m3 grid and within one grid step of... the rounded exact logit is
+    # not available here; what is: rows still sum to one
+    ones = oracle.run_all(q, k, torch.ones_like(v), scale=sc, flags=oracle.SR_E4M3, sr_seed=11)
+    assert np.abs(ones.out - 1.0).max() < 1e-6
+
+
 def test_overflow_rule_of_section_3_3():
     f = GOLD["logit_bound_factor"]
     assert abs(f - 8 * math.sqrt(2)) < 1e-12
