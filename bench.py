@@ -7,7 +7,7 @@ input (B=4, 32 query / 8 KV heads, N=8192, head_dim 128, causal).  Prints ONE JS
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config C]
                   [--mode lamp|force8|force16] [--tau T] [--delta D] [--no-stage1]
-                  [--compact] [--h16-seq] [--scale-mult M] [--window W]
+                  [--compact] [--h16-seq] [--sr] [--scale-mult M] [--window W]
 
 The options after --config select the other workloads and the paper's ablations (threshold
 and margin sweeps, stage 1 off, the scale sweep of the long-context config, the sliding
@@ -131,7 +131,8 @@ def oracle_sample_run(cfg, q, k, v, scale, n_units, seed=11, knobs=None):
     units = li.sample_units(cfg, n_units, seed=seed)
     t0 = time.perf_counter()
     oracle.run_units(q, k, v, units, scale=scale, causal=cfg.causal, window=window, tau=kn.get("tau", 0.5),
-                     delta=kn.get("delta", 2.0 ** -8), flags=kn.get("flags", 0), checksums=False)
+                     delta=kn.get("delta", 2.0 ** -8), flags=kn.get("flags", 0), sr_seed=kn.get("sr_seed", 0),
+                     checksums=False)
     dt = time.perf_counter() - t0
     fl = sum(4.0 * cfg.D * unit_pairs(cfg, int(g), window) for _, _, g in units)
     return dt, fl, len(units)
@@ -139,8 +140,8 @@ def oracle_sample_run(cfg, q, k, v, scale, n_units, seed=11, knobs=None):
 
 def knobs_of(args):
     """Thresholds, mode bits and mask of this run (the same numeric flag values in the library and the oracle)."""
-    flags = {"lamp": 0, "force8": 2, "force16": 1}[args.mode] | (4 if args.no_stage1 else 0) | (16 if args.compact else 0) | (32 if args.h16_seq else 0)
-    return {"tau": args.tau, "delta": args.delta, "flags": flags, "window": args.window}
+    flags = {"lamp": 0, "force8": 2, "force16": 1}[args.mode] | (4 if args.no_stage1 else 0) | (16 if args.compact else 0) | (32 if args.h16_seq else 0) | (64 if args.sr else 0)
+    return {"tau": args.tau, "delta": args.delta, "flags": flags, "window": args.window, "sr_seed": args.sr_seed}
 
 
 def reference_arm(args, cfg, rank):
@@ -186,6 +187,8 @@ def workload_config(cfg, args):
         extra += ", compact-layout branch"
     if args.h16_seq:
         extra += ", per-step e4m11 accumulation"
+    if args.sr:
+        extra += f", stochastic rounding (seed {args.sr_seed})"
     return {"workload": f"config {cfg.index}: {cfg.name} prefill, B={cfg.B}, Hq={cfg.Hq}, Hkv={cfg.Hkv}, "
                         f"N={cfg.N}, head_dim={cfg.D}, causal{extra}, tau={args.tau:g}, delta=2^{math.log2(args.delta):g}",
             "l2": "inputs (Q+K+V+O = %.0f MB) larger than the 126 MB L2" %
@@ -209,6 +212,9 @@ def main():
                     help="the compact register layout's branch: two or more marked sub-blocks send the tile to 16 bits")
     ap.add_argument("--h16-seq", action="store_true",
                     help="16-bit logits by per-step e4m11 accumulation (the other reading of the 16-bit accumulate)")
+    ap.add_argument("--sr", action="store_true",
+                    help="stochastic rounding in the 8-bit accumulation (Sec. 3.3), counter-based generator")
+    ap.add_argument("--sr-seed", type=int, default=1)
     ap.add_argument("--scale-mult", type=float, default=1.0, help="softmax scale = mult / sqrt(head_dim)")
     ap.add_argument("--window", type=int, default=0, help="sliding window (0 = global causal)")
     args = ap.parse_args()
@@ -250,7 +256,7 @@ def main():
     p.batch, p.heads_q, p.heads_kv, p.seqlen, p.head_dim = B, Hq, k.shape[1], N, D
     lamp.lamp_attn_contiguous_strides(p)
     p.causal, p.window, p.scale = 1, args.window, scale
-    p.threshold, p.delta, p.flags = args.tau, args.delta, kn["flags"]
+    p.threshold, p.delta, p.flags, p.sr_seed = args.tau, args.delta, kn["flags"], args.sr_seed
     fl = flops_of(cfg, args.window)
 
     def step():
@@ -312,7 +318,7 @@ def main():
     peak = 4.0 / MIN_SLOTS_PER_STEP * SM_COUNT * LANES_PER_SM * SM_MAX_MHZ * 1e6 / 1e12
     # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu capture summarised in
     # profiles/lamp_fwd_sm100_config2_ncu_full.txt (algorithmic bytes: 680 MB)
-    headline = (args.mode == "lamp" and not args.no_stage1 and not args.compact and not args.h16_seq and args.tau == 0.5 and args.delta == 2.0 ** -8
+    headline = (args.mode == "lamp" and not args.no_stage1 and not args.compact and not args.h16_seq and not args.sr and args.tau == 0.5 and args.delta == 2.0 ** -8
                 and args.scale_mult == 1.0 and args.window == 0)
     traffic = {2: 655.97e6}.get(cfg.index) if headline else None
     roofline = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",

@@ -59,6 +59,15 @@ typedef enum lamp_attn_error {
                                       product rounded once (the library's default reading of the 16-bit
                                       accumulation); much slower on this GPU, for comparison only          */
 
+#define LAMP_SR_E4M3         0x40u /* stochastic instead of nearest-even rounding in the 8-bit accumulation, which
+                                      Sec. 3.3 proposes against swamping.  Rule (integer arithmetic, so that two
+                                      implementations agree bit for bit): the fp32 bit pattern of the magnitude plus
+                                      a uniform 20-bit integer, low 20 mantissa bits cleared; magnitudes below 2^-6
+                                      are moved into [2^-6, 2^-5) by one fp32 addition first and back afterwards;
+                                      beyond 448 saturates.  The 20 bits of a step are a 32-bit integer hash of
+                                      (sr_seed, batch * heads_q + head, query row, key, channel).  About seven
+                                      times the work per step; not combinable with LAMP_H16_SEQ               */
+
 typedef struct lamp_attn_params {
   int32_t batch, heads_q, heads_kv; /* heads_q % heads_kv == 0 (grouped-query attention)      */
   int32_t seqlen;                   /* multiple of 128                                         */
@@ -81,6 +90,8 @@ typedef struct lamp_attn_params {
                                        those replaced in stage 2), 0xFF elsewhere             */
   uint64_t* dbg_checksums;          /* [batch, heads_q, seqlen/32, seqlen/64, 2]: position-keyed
                                        checksums of the y8 and e8 bytes of each (group, tile)  */
+  uint32_t sr_seed;                 /* seed of the generator of LAMP_SR_E4M3 (unused otherwise)  */
+  uint32_t reserved;                /* set to 0                                                  */
 } lamp_attn_params;
 
 /* Counters of the most recent lamp_attn_fwd on the current device. */

@@ -1,0 +1,100 @@
+"""Output error of the forward pass against exact (fp64) softmax attention, per mode.
+
+    python -m paper_2609_39361_b200.accuracy [--config C] [--heads H] [--seqlen N]
+
+The paper's tables report downstream task metrics of real models; those need weights and
+datasets.  What can be measured on the synthetic inputs is the quantity the method controls:
+how far the attention output moves from the exact one, for the pure 8-bit pass, LAMP at the
+paper's thresholds, the all-16-bit pass, and the optional modes.  Prints one JSON line per mode
+with the relative Frobenius error of O, the largest absolute error of O and of lse, and the
+recomputed share.  The reference is plain fp64 torch arithmetic on the GPU, one head at a time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+
+import torch
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+sys.path.insert(0, ROOT)
+
+import lamp_inputs as li  # noqa: E402
+import paper_2609_39361_b200 as lamp  # noqa: E402
+
+
+def exact_attention(q, k, v, scale, window=0):
+    """fp64 causal softmax attention; q [B, Hq, N, D], k / v [B, Hkv, N, D] on the GPU."""
+    B, Hq, N, D = q.shape
+    rep = Hq // k.shape[1]
+    out = torch.empty(B, Hq, N, D, dtype=torch.float64, device=q.device)
+    lse = torch.empty(B, Hq, N, dtype=torch.float64, device=q.device)
+    i = torch.arange(N, device=q.device)[None, :]
+    j = torch.arange(N, device=q.device)[:, None]
+    mask = i > j
+    if window:
+        mask |= (j - i) >= window
+    # the library folds the scale into Q in fp32 before anything else; the exact reference does not round
+    for b in range(B):
+        for h in range(Hq):
+            s = (q[b, h].double() @ k[b, h // rep].double().T) * float(scale)
+            s.masked_fill_(mask, float("-inf"))
+            lse[b, h] = torch.logsumexp(s, -1)
+            out[b, h] = torch.softmax(s, -1) @ v[b, h // rep].double()
+    return out, lse
+
+
+MODES = [
+    ("force8", lamp.LAMP_FORCE_8BIT, {}),
+    ("lamp", 0, {}),
+    ("lamp tau=2^-3", 0, {"threshold": 0.125}),
+    ("lamp delta=2^-4", 0, {"delta": 2.0 ** -4}),
+    ("lamp stage 1 off", lamp.LAMP_NO_STAGE1, {}),
+    ("lamp compact branch", lamp.LAMP_COMPACT_BRANCH, {}),
+    ("lamp per-step e4m11", lamp.LAMP_H16_SEQ, {}),
+    ("force16", lamp.LAMP_FORCE_16BIT, {}),
+    ("force8 stochastic", lamp.LAMP_FORCE_8BIT | lamp.LAMP_SR_E4M3, {"sr_seed": 1}),
+    ("lamp stochastic", lamp.LAMP_SR_E4M3, {"sr_seed": 1}),
+]
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--config", type=int, default=1)
+    ap.add_argument("--heads", type=int, default=0, help="query heads to keep (0 = all of the config)")
+    ap.add_argument("--seqlen", type=int, default=0, help="sequence length (0 = the config's)")
+    ap.add_argument("--scale-mult", type=float, default=1.0)
+    ap.add_argument("--window", type=int, default=0)
+    args = ap.parse_args()
+    if not torch.cuda.is_available():
+        raise SystemExit("needs a CUDA device")
+    cfg = li.CONFIGS[args.config]
+    kw = {}
+    if args.heads:
+        kw.update(Hq=args.heads, Hkv=max(1, args.heads * cfg.Hkv // cfg.Hq))
+    if args.seqlen:
+        kw.update(N=args.seqlen)
+    q, k, v = li.make_qkv(cfg, **kw)
+    dev = torch.device("cuda:0")
+    q, k, v = q.to(dev), k.to(dev), v.to(dev)
+    scale = li.softmax_scale(cfg.D, args.scale_mult)
+    ref_o, ref_l = exact_attention(q, k, v, scale, args.window)
+    for name, flags, extra in MODES:
+        r = lamp.forward(q, k, v, scale=scale, window=args.window, flags=flags, out_fp32=True, **extra)
+        st = lamp.lamp_attn_get_stats()
+        o = r["out"].double()
+        line = {"mode": name, "config": f"{cfg.name} B={q.shape[0]} Hq={q.shape[1]} N={q.shape[2]} D={q.shape[3]}",
+                "rel_fro_err_out": float((o - ref_o).norm() / ref_o.norm()),
+                "max_abs_err_out": float((o - ref_o).abs().max()),
+                "max_abs_err_lse": float((r["lse"].double() - ref_l).abs().max()),
+                "recomputed_subblock_pct": 100.0 * (st["stage1_flagged"] + st["stage2_flagged"]) /
+                                           max(st["subblocks_active"], 1),
+                "exp16_above_one": st["exp16_gt1"], "saturated_e4m3": st["sat_e4m3"],
+                "saturated_e4m11": st["sat_e4m11"]}
+        print(json.dumps(line))
+
+
+if __name__ == "__main__":
+    main()

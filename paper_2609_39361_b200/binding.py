@@ -7,7 +7,7 @@ import os
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "liblamp_attn.so")
 
-LAMP_FORCE_16BIT, LAMP_FORCE_8BIT, LAMP_NO_STAGE1, LAMP_OUT_FP32, LAMP_COMPACT_BRANCH, LAMP_H16_SEQ = 1, 2, 4, 8, 16, 32
+LAMP_FORCE_16BIT, LAMP_FORCE_8BIT, LAMP_NO_STAGE1, LAMP_OUT_FP32, LAMP_COMPACT_BRANCH, LAMP_H16_SEQ, LAMP_SR_E4M3 = 1, 2, 4, 8, 16, 32, 64
 
 EXPORTS = ("lamp_attn_default_params", "lamp_attn_contiguous_strides", "lamp_attn_workspace_bytes",
            "lamp_attn_fwd", "lamp_attn_fwd_digest", "lamp_attn_debug_round_e4m3", "lamp_attn_get_stats", "lamp_attn_last_cuda_error", "lamp_attn_strerror")
@@ -25,7 +25,8 @@ class LampAttnParams(C.Structure):
                 ("causal", C.c_int32), ("window", C.c_int32), ("scale", C.c_float),
                 ("threshold", C.c_float), ("delta", C.c_float), ("flags", C.c_uint32),
                 ("dbg_batch", C.c_int32), ("dbg_head", C.c_int32),
-                ("dbg_y8", C.c_void_p), ("dbg_e8", C.c_void_p), ("dbg_checksums", C.c_void_p)]
+                ("dbg_y8", C.c_void_p), ("dbg_e8", C.c_void_p), ("dbg_checksums", C.c_void_p),
+                ("sr_seed", C.c_uint32), ("reserved", C.c_uint32)]
 
 
 class LampAttnStats(C.Structure):
@@ -150,7 +151,7 @@ def lamp_attn_get_stats(stream=None) -> dict:
     return st.as_dict()
 
 
-def forward(q, k, v, *, causal=True, window=0, scale=None, threshold=0.5, delta=2.0 ** -8, flags=0,
+def forward(q, k, v, *, causal=True, window=0, scale=None, threshold=0.5, delta=2.0 ** -8, flags=0, sr_seed=0,
             out_fp32=False, want_lse=True, want_flags=True, dump=None, checksums=False, stream=None):
     """Convenience wrapper: allocate outputs with torch, fill the params struct, call
     ``lamp_attn_fwd``.  q: [B, Hq, N, D] bf16 CUDA; k, v: [B, Hkv, N, D].
@@ -169,6 +170,7 @@ def forward(q, k, v, *, causal=True, window=0, scale=None, threshold=0.5, delta=
     p.scale = float(scale) if scale is not None else float(torch.tensor(D, dtype=torch.float64).rsqrt().float())
     p.threshold, p.delta = float(threshold), float(delta)
     p.flags = int(flags) | (LAMP_OUT_FP32 if out_fp32 else 0)
+    p.sr_seed = int(sr_seed)
     res = {"out": out}
     lse = torch.empty(B, Hq, N, device=q.device, dtype=torch.float32) if want_lse else None
     fm = torch.empty(B, Hq, N // 32, N // 64, device=q.device, dtype=torch.uint8) if want_flags else None

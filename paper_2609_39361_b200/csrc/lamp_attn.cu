@@ -94,12 +94,14 @@ static int ensure_device(int* dev_out) {
     if (!fn || qr != cudaDriverEntryPointSuccess) return cuda_fail(cudaErrorNotSupported);
     g_encode = (TensorMapEncodeFn)fn;
   }
-  const void* kernels[8] = {
-      (const void*)lamp_fwd_sm100<128, false, false>, (const void*)lamp_fwd_sm100<128, true, false>,
-      (const void*)lamp_fwd_sm100<256, false, false>, (const void*)lamp_fwd_sm100<256, true, false>,
-      (const void*)lamp_fwd_sm100<128, false, true>,  (const void*)lamp_fwd_sm100<128, true, true>,
-      (const void*)lamp_fwd_sm100<256, false, true>,  (const void*)lamp_fwd_sm100<256, true, true>};
-  for (int i = 0; i < 8; ++i) {
+  const void* kernels[12] = {
+      (const void*)lamp_fwd_sm100<128, false, 0>, (const void*)lamp_fwd_sm100<128, true, 0>,
+      (const void*)lamp_fwd_sm100<256, false, 0>, (const void*)lamp_fwd_sm100<256, true, 0>,
+      (const void*)lamp_fwd_sm100<128, false, 1>, (const void*)lamp_fwd_sm100<128, true, 1>,
+      (const void*)lamp_fwd_sm100<256, false, 1>, (const void*)lamp_fwd_sm100<256, true, 1>,
+      (const void*)lamp_fwd_sm100<128, false, 2>, (const void*)lamp_fwd_sm100<128, true, 2>,
+      (const void*)lamp_fwd_sm100<256, false, 2>, (const void*)lamp_fwd_sm100<256, true, 2>};
+  for (int i = 0; i < 12; ++i) {
     e = cudaFuncSetAttribute(kernels[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLaunch);
     if (e != cudaSuccess) return cuda_fail(e);
   }
@@ -166,10 +168,11 @@ static int check_params(const void* q, const void* k, const void* v, void* out,
   if (p->heads_q % p->heads_kv) return LAMP_ERR_INVALID_ARG;
   if (!(p->threshold >= 0.0f) || !(p->delta >= 0.0f) || !isfinite(p->scale)) return LAMP_ERR_INVALID_ARG;
   if (p->window < 0 || (p->window > 0 && !p->causal)) return LAMP_ERR_INVALID_ARG;
-  if (p->flags & ~(LAMP_FORCE_16BIT | LAMP_FORCE_8BIT | LAMP_NO_STAGE1 | LAMP_OUT_FP32 | LAMP_COMPACT_BRANCH | LAMP_H16_SEQ))
+  if (p->flags & ~(LAMP_FORCE_16BIT | LAMP_FORCE_8BIT | LAMP_NO_STAGE1 | LAMP_OUT_FP32 | LAMP_COMPACT_BRANCH | LAMP_H16_SEQ | LAMP_SR_E4M3))
     return LAMP_ERR_INVALID_ARG;
   if ((p->flags & LAMP_FORCE_16BIT) && (p->flags & (LAMP_FORCE_8BIT | LAMP_NO_STAGE1)))
     return LAMP_ERR_INVALID_ARG;
+  if ((p->flags & LAMP_SR_E4M3) && (p->flags & LAMP_H16_SEQ)) return LAMP_ERR_INVALID_ARG;
   if ((p->dbg_y8 || p->dbg_e8) &&
       (p->dbg_batch < 0 || p->dbg_batch >= p->batch || p->dbg_head < 0 || p->dbg_head >= p->heads_q))
     return LAMP_ERR_INVALID_ARG;
@@ -204,7 +207,7 @@ int lamp_attn_fwd(const void* q, const void* k, const void* v, void* out, float*
   }
   P.batch = p->batch; P.heads_q = p->heads_q; P.heads_kv = p->heads_kv; P.seqlen = p->seqlen;
   P.causal = p->causal ? 1 : 0; P.window = p->window;
-  P.scale = p->scale; P.tau = p->threshold; P.delta = p->delta; P.flags = p->flags;
+  P.scale = p->scale; P.tau = p->threshold; P.delta = p->delta; P.flags = p->flags; P.sr_seed = p->sr_seed;
   P.dbg_batch = p->dbg_batch; P.dbg_head = p->dbg_head;
   P.dbg_y8 = p->dbg_y8; P.dbg_e8 = p->dbg_e8;
   P.dbg_checksums = (unsigned long long*)p->dbg_checksums;
@@ -236,16 +239,22 @@ int lamp_attn_fwd(const void* q, const void* k, const void* v, void* out, float*
   dim3 grid(p->seqlen / kBM, p->heads_q, p->batch), block(kThreads);
   const uint2* lutp = (const uint2*)lut_ptr;
   DeviceStats* dsp = (DeviceStats*)stats_ptr;
-#define LAMP_LAUNCH(D_, DUMP_, SEQ_) \
-  lamp_fwd_sm100<D_, DUMP_, SEQ_><<<grid, block, kSmemLaunch, stream>>>(P, kmap, vmap, lutp, dsp)
-  const bool seq16 = (p->flags & LAMP_H16_SEQ) != 0;   // the per-step 16-bit accumulation has kernels of its own
+#define LAMP_LAUNCH(D_, DUMP_, VAR_) \
+  lamp_fwd_sm100<D_, DUMP_, VAR_><<<grid, block, kSmemLaunch, stream>>>(P, kmap, vmap, lutp, dsp)
+#define LAMP_LAUNCH_VAR(D_, DUMP_)                  \
+  do {                                              \
+    if (var == 0) LAMP_LAUNCH(D_, DUMP_, 0);        \
+    else if (var == 1) LAMP_LAUNCH(D_, DUMP_, 1);   \
+    else LAMP_LAUNCH(D_, DUMP_, 2);                 \
+  } while (0)
+  // the per-step 16-bit accumulation (1) and the stochastic rounding (2) have kernels of their own
+  const int var = (p->flags & LAMP_H16_SEQ) ? 1 : (p->flags & LAMP_SR_E4M3) ? 2 : 0;
   if (p->head_dim == 128) {
-    if (seq16) { if (dump) LAMP_LAUNCH(128, true, true); else LAMP_LAUNCH(128, false, true); }
-    else       { if (dump) LAMP_LAUNCH(128, true, false); else LAMP_LAUNCH(128, false, false); }
+    if (dump) LAMP_LAUNCH_VAR(128, true); else LAMP_LAUNCH_VAR(128, false);
   } else {
-    if (seq16) { if (dump) LAMP_LAUNCH(256, true, true); else LAMP_LAUNCH(256, false, true); }
-    else       { if (dump) LAMP_LAUNCH(256, true, false); else LAMP_LAUNCH(256, false, false); }
+    if (dump) LAMP_LAUNCH_VAR(256, true); else LAMP_LAUNCH_VAR(256, false);
   }
+#undef LAMP_LAUNCH_VAR
 #undef LAMP_LAUNCH
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);

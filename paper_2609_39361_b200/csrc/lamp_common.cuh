@@ -74,6 +74,27 @@ __device__ __forceinline__ float rne_e4m11(double x) {
   return copysignf((float)r, (float)x);
 }
 
+// Stochastic rounding onto the e4m3 grid with a uniform 20-bit integer u (mode LAMP_SR_E4M3): bit pattern of
+// the magnitude plus u, low 20 mantissa bits cleared; the subnormal range (spacing 2^-9 below 2^-6) is
+// handled inside [2^-6, 2^-5), which has that spacing; saturating at 448.
+__device__ __forceinline__ float sr_e4m3(float t, uint32_t u) {
+  const float a = fabsf(t);
+  const float off = a < 0.015625f ? 0.015625f : 0.0f;
+  const float s = __fadd_rn(a, off);
+  const uint32_t bits = (__float_as_uint(s) + u) & 0xFFF00000u;
+  const float r = fminf(__fsub_rn(__uint_as_float(bits), off), 448.0f);
+  return copysignf(r, t);
+}
+// The 20 random bits of one accumulation step: a 32-bit integer hash of its coordinates, already
+// combined by the caller into x = seed ^ bh*c0 ^ row*c1 ^ key*c2 ^ channel*c3.
+constexpr uint32_t kSrMulBh = 0x27D4EB2Fu, kSrMulRow = 0x85EBCA77u, kSrMulKey = 0x9E3779B1u, kSrMulCh = 0xC2B2AE3Du;
+__device__ __forceinline__ uint32_t sr_bits(uint32_t x) {
+  x ^= x >> 16; x *= 0x7FEB352Du;
+  x ^= x >> 15; x *= 0x846CA68Bu;
+  x ^= x >> 16;
+  return x >> 12;
+}
+
 // The same rounding of an fp32 value (the per-step 16-bit accumulation mode).
 __device__ __forceinline__ float rne_e4m11_f(float t) {
   const float a = fabsf(t);
@@ -139,6 +160,7 @@ struct KernelParams {
   int causal, window;
   float scale, tau, delta;
   uint32_t flags;
+  uint32_t sr_seed;
   int dbg_batch, dbg_head;
   uint8_t* dbg_y8;
   uint8_t* dbg_e8;

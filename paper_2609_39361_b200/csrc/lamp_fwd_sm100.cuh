@@ -136,6 +136,51 @@ __device__ __forceinline__ void chain8(const void* __restrict__ q, const float* 
   }
 }
 
+// The first pass with stochastic rounding (mode LAMP_SR_E4M3): the same recursion, scalar FMAs, each
+// step rounded with 20 bits drawn from the hash of (seed, head, query row, key, channel).
+// row_key[a]: seed ^ bh*c0 ^ row_a*c1 for the lane's four query rows; key0: the lane's first key times c2;
+// ch0: first channel of this call.  A comparison mode, not tuned.
+template <bool QF32, bool FIRST>
+__device__ __forceinline__ void chain8_sr(const void* __restrict__ q, const float* __restrict__ kf, float scale,
+                                          float (&acc)[4][16], const uint32_t (&row_key)[4], uint32_t key0, int ch0) {
+  if (FIRST) {
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+      for (int b = 0; b < 16; ++b) acc[a][b] = 0.0f;
+  }
+  const float* qf = reinterpret_cast<const float*>(q);
+  const __nv_bfloat16* qh = reinterpret_cast<const __nv_bfloat16*>(q);
+#pragma unroll 1
+  for (int kk = 0; kk < kHalf; ++kk) {
+    float q4[4];
+    if (QF32) {
+      const float4 qv = *reinterpret_cast<const float4*>(qf + kk * kBM);
+      q4[0] = qv.x; q4[1] = qv.y; q4[2] = qv.z; q4[3] = qv.w;
+    } else {
+      const uint2 qv = *reinterpret_cast<const uint2*>(qh + kk * kBM);
+      q4[0] = __fmul_rn(__uint_as_float(qv.x << 16), scale);
+      q4[1] = __fmul_rn(__uint_as_float(qv.x & 0xffff0000u), scale);
+      q4[2] = __fmul_rn(__uint_as_float(qv.y << 16), scale);
+      q4[3] = __fmul_rn(__uint_as_float(qv.y & 0xffff0000u), scale);
+    }
+    const uint32_t chx = (uint32_t)(ch0 + kk) * kSrMulCh;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const float4 kv4 = *reinterpret_cast<const float4*>(kf + kk * kKfStride + 4 * c);
+      const float kv[4] = {kv4.x, kv4.y, kv4.z, kv4.w};
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int b = 4 * c + u;
+        const uint32_t kx = (key0 + (uint32_t)b * kSrMulKey) ^ chx;
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+          acc[a][b] = sr_e4m3(__fmaf_rn(kv[u], q4[a], acc[a][b]), sr_bits(row_key[a] ^ kx));
+      }
+    }
+  }
+}
+
 // 16-bit logits of one sub-block for this lane's (quad x 4 keys): a sequential fp64 fma
 // chain over kk, scaled, rounded once to e4m11, stored to TMEM columns tdst..tdst+15.
 // The fp32 -> fp64 conversions are the slow part on this GPU (they hold the scheduler for
@@ -332,7 +377,7 @@ __device__ __forceinline__ uint32_t enc_exp8(float e) {
 // The 64 first-pass logits of a lane arrive packed in 16 words (yw) and are unpacked 16 at a
 // time, so that the per-element work is a short loop instead of a long unrolled stretch of
 // code and the registers are free for the 16-bit path.
-template <int D, bool FULL, bool DUMP, bool SEQ16>
+template <int D, bool FULL, bool DUMP, int VAR>
 __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileGeom& g, const uint32_t (&yw)[16],
                                               const __nv_bfloat16* ktile, int64_t kstride, uint32_t tq,
                                               const uint2* lut, double* dscr, unsigned char* phi, unsigned char* plo,
@@ -348,7 +393,7 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
   const bool skip1 = (P.flags & (LAMP_FORCE_8BIT | LAMP_NO_STAGE1)) != 0;
   auto logits16 = [&](int th) {
     const __nv_bfloat16* kr = ktile + (int64_t)(16 * th) * kstride;
-    if constexpr (SEQ16) dot16_seq<D>(kr, kstride, q_quad, P.scale, tscratch + 16 * th);
+    if constexpr (VAR == 1) dot16_seq<D>(kr, kstride, q_quad, P.scale, tscratch + 16 * th);
     else dot16<D>(kr, kstride, tq, dscr, scale_d, tscratch + 16 * th);
   };
 
@@ -760,9 +805,10 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
 }
 
 
-// SEQ16: the per-step reading of the 16-bit accumulation (mode LAMP_H16_SEQ), a kernel of its own so that
-// the default one carries nothing of it (code that never ran still cost it 2.5 % through register allocation).
-template <int D, bool DUMP, bool SEQ16>
+// VAR 1: the per-step reading of the 16-bit accumulation (mode LAMP_H16_SEQ); VAR 2: stochastic rounding in
+// the first pass (mode LAMP_SR_E4M3).  Kernels of their own, so that the default one (VAR 0) carries nothing
+// of them (code that never ran still cost it 2.5 % through register allocation).
+template <int D, bool DUMP, int VAR>
 __global__ void __launch_bounds__(kThreads, 1)
 lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ CUtensorMap kmap,
                const __grid_constant__ CUtensorMap vmap, const uint2* __restrict__ lut_g,
@@ -983,8 +1029,18 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
         ok = ok && ptx::mbar_wait(&bars[kKfFull0 + (m & 3)], (m >> 2) & 1, status, kTimeoutCode);
         if (any) {
           const unsigned char* qh = q_quad + (size_t)hh * kHalf * kBM * (QF32 ? 4 : 2);
-          if (hh == 0) chain8<QF32, true>(qh, kf, P.scale, acc);
-          else chain8<QF32, false>(qh, kf, P.scale, acc);
+          if constexpr (VAR == 2) {
+            uint32_t row_key[4];
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+              row_key[a] = P.sr_seed ^ ((uint32_t)(b * P.heads_q + h) * kSrMulBh) ^ ((uint32_t)(j0 + 4 * qa + a) * kSrMulRow);
+            const uint32_t key0 = (uint32_t)(i0 + 16 * (lane & 3)) * kSrMulKey;
+            if (hh == 0) chain8_sr<QF32, true>(qh, kf, P.scale, acc, row_key, key0, hh * kHalf);
+            else chain8_sr<QF32, false>(qh, kf, P.scale, acc, row_key, key0, hh * kHalf);
+          } else {
+            if (hh == 0) chain8<QF32, true>(qh, kf, P.scale, acc);
+            else chain8<QF32, false>(qh, kf, P.scale, acc);
+          }
         }
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&bars[kKfEmpty0 + (m & 3)]);
@@ -1018,7 +1074,7 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
     const bool dump_rows = DUMP && b == P.dbg_batch && h == P.dbg_head;
     const __nv_bfloat16* kg = P.k + b * P.ks[0] + hk * P.ks[1];
     double* dscr = dscr_all + grp * 384;
-    const unsigned char* q_quad = SEQ16 ? qs + (QF32 ? 4 : 2) * (grp * kBQ + 4 * qa) : nullptr;
+    const unsigned char* q_quad = VAR == 1 ? qs + (QF32 ? 4 : 2) * (grp * kBQ + 4 * qa) : nullptr;
     const uint32_t tlane = tbase + ((uint32_t)(grp * 32) << 16);
     const uint32_t tscr = tlane + kColScr, tq = tlane + kColQ, tring = tlane + kColRing;
     {
@@ -1084,11 +1140,11 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
         const int dump0 = dump_rows ? j0 : -1;
         const __nv_bfloat16* ktile = kg + (int64_t)i0 * P.ks[2];
         if (full)
-          flag = lamp_post<D, true, DUMP, SEQ16>(P, g, yw, ktile, P.ks[2], tq, lut, dscr, phi, plo, tscr, lo_dirty,
+          flag = lamp_post<D, true, DUMP, VAR>(P, g, yw, ktile, P.ks[2], tq, lut, dscr, phi, plo, tscr, lo_dirty,
                                           st, lam, wc, cks, dump0, grp * kBQ, ph, &bars[kPvDone0 + grp], (n - 1) & 1, n > 0,
                                           status, ok, q_quad);
         else
-          flag = lamp_post<D, false, DUMP, SEQ16>(P, g, yw, ktile, P.ks[2], tq, lut, dscr, phi, plo, tscr, lo_dirty,
+          flag = lamp_post<D, false, DUMP, VAR>(P, g, yw, ktile, P.ks[2], tq, lut, dscr, phi, plo, tscr, lo_dirty,
                                            st, lam, wc, cks, dump0, grp * kBQ, ph, &bars[kPvDone0 + grp], (n - 1) & 1, n > 0,
                                            status, ok, q_quad);
       } else {

@@ -32,5 +32,5 @@ def test_host_only_calls_work_without_a_device():
 
 def test_struct_layout_matches_header():
     import ctypes as C
-    assert C.sizeof(lamp.LampAttnParams) == 176
+    assert C.sizeof(lamp.LampAttnParams) == 184
     assert C.sizeof(lamp.LampAttnStats) == 168

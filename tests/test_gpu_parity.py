@@ -95,6 +95,23 @@ def test_threshold_and_margin_sweeps(flags, tau, delta):
     compare_dense_bytes(gpu, ref, 0, 1)
 
 
+@pytest.mark.parametrize("flags,seed,D", [(oracle.SR_E4M3, 1, 128), (oracle.SR_E4M3, 0xdeadbeef, 128),
+                                          (oracle.SR_E4M3 | oracle.FORCE_8BIT, 7, 128),
+                                          (oracle.SR_E4M3 | oracle.COMPACT_BRANCH, 3, 128), (oracle.SR_E4M3, 5, 256)])
+def test_stochastic_rounding_of_the_first_pass(flags, seed, D):
+    """Stochastic rounding in the 8-bit accumulation (Sec. 3.3): both sides draw the same 20 bits per step
+    from the counter-based generator, so the first-pass bytes and everything after them agree exactly."""
+    cfg = li.CONFIGS[1 if D == 128 else 3]
+    q, k, v = li.make_qkv(cfg, B=1, Hq=2, Hkv=1, N=384, seed=41)
+    sc = li.softmax_scale(cfg.D)
+    ref = oracle.run_all(q, k, v, scale=sc, flags=flags, sr_seed=seed, dumps=True)
+    gpu = run_gpu(q, k, v, scale=sc, flags=flags, sr_seed=seed, dump=(0, 1))
+    compare_units(gpu, ref, check_stats=True, label=f"sr flags={flags} seed={seed} D={D}")
+    compare_dense_bytes(gpu, ref, 0, 1)
+    plain = oracle.run_all(q, k, v, scale=sc, flags=flags & ~oracle.SR_E4M3, dumps=True)
+    assert not np.array_equal(plain.y8, ref.y8)
+
+
 @pytest.mark.parametrize("window,flags", [(0, 0), (192, 0), (0, oracle.FORCE_16BIT), (0, oracle.H16_SEQ)])
 def test_head_dim_256_gemma_shaped(window, flags):
     """head_dim 256 (two 128-channel halves per tile), global and sliding-window layers."""
