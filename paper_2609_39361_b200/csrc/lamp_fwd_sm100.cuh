@@ -181,11 +181,25 @@ __device__ __forceinline__ void chain8_sr(const void* __restrict__ q, const floa
   }
 }
 
+// D (8 x 8) += A (8 x 4) B (4 x 8) in fp64 on the tensor core.  Lane l = 4g + t holds A[g][t], B[t][g],
+// D[g][2t], D[g][2t+1].  Measured on B200: bit-identical to four chained fma in ascending k (against a
+// CPU chain on operands whose exponents spread over 2^60, where any other order differs), 16 cycles per
+// instruction = the rate of the 8 DFMA per lane it replaces, for one issue slot instead of eight.
+__device__ __forceinline__ void dmma_884(double& d0, double& d1, double a, double b) {
+  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
+               : "+d"(d0), "+d"(d1) : "d"(a), "d"(b));
+}
+
 // 16-bit logits of one sub-block for this lane's (quad x 4 keys): a sequential fp64 fma
 // chain over kk, scaled, rounded once to e4m11, stored to TMEM columns tdst..tdst+15.
-// The fp32 -> fp64 conversions are the slow part on this GPU (they hold the scheduler for
-// several cycles each), so the warp converts each operand once per 8 channels into a small
-// shared-memory scratch (16 keys and 32 rows as doubles) and every lane reads from there.
+// The chain runs on the fp64 tensor-core instruction, four channels per instruction in ascending
+// order, which keeps the sequential rounding of the chain bit for bit.  Rows and keys are assigned to
+// the instruction's tiles so that a lane ends with exactly its own 4 queries x 4 keys: tile row
+// (mt, g) is query 4g + mt, tile column (nt, 2t + e) is key 4t + 2nt + e.
+// The fp32 -> fp64 conversions are slow on this GPU (they hold the scheduler for several cycles each),
+// so the warp converts each operand once per 8 channels into a small shared-memory scratch (16 keys
+// and 32 rows as doubles, columns swizzled by the channel so that the fragment loads of lanes with
+// different t fall into different banks) and every lane reads its fragments from there.
 // krow: global bf16 row of the sub-block's first key (lane l fetches key l % 16, channels
 // 4 (l / 16) .. +3 of every 8; the rows were just streamed through L2 by TMA).
 // tq: TMEM columns holding the query row of this lane (row = lane of the group).  head_dim 128:
@@ -197,19 +211,20 @@ __device__ __noinline__ void dot16(const __nv_bfloat16* __restrict__ krow, int64
                                    double* dscr, double scale_d, uint32_t tdst) {
   constexpr bool QHI = (D == 128);
   constexpr int QW = QHI ? 8 : 4;   // TMEM columns per 8 channels
-  const int lane = threadIdx.x & 31, qa = lane >> 2, tp = lane & 3;
+  const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   __builtin_assume(__isShared(dscr));
   double* kscr = dscr;          // [8 kk][16 keys]
   double* qscr = dscr + 128;    // [8 kk][32 rows]
   uint32_t* khi = reinterpret_cast<uint32_t*>(kscr) + 1;   // high words of the same
   uint32_t* qhi = reinterpret_cast<uint32_t*>(qscr) + 1;
-  double acc[4][4];
+  double acc[4][2][2];          // [mt][nt][e]: query 4g + mt, key 4t + 2nt + e
 #pragma unroll
-  for (int a = 0; a < 4; ++a)
+  for (int mt = 0; mt < 4; ++mt)
 #pragma unroll
-    for (int b = 0; b < 4; ++b) acc[a][b] = 0.0;
+    for (int nt = 0; nt < 2; ++nt) acc[mt][nt][0] = acc[mt][nt][1] = 0.0;
   const int kh = lane >> 4;      // which four of a chunk's eight channels this lane converts for K
-  const __nv_bfloat16* ksrc = krow + (int64_t)(lane & 15) * kstride + 4 * kh;
+  const int key = lane & 15;
+  const __nv_bfloat16* ksrc = krow + (int64_t)key * kstride + 4 * kh;
   uint2 kraw = *reinterpret_cast<const uint2*>(ksrc);
   uint32_t qraw[QW];
   auto fetch_q = [&](int k0) {
@@ -221,6 +236,14 @@ __device__ __noinline__ void dot16(const __nv_bfloat16* __restrict__ krow, int64
       qraw[0] = v.x; qraw[1] = v.y; qraw[2] = v.z; qraw[3] = v.w;
     }
   };
+  // fragment addresses of this lane inside one 4-channel step (channel = 4 ks + t of the chunk)
+  const int qsw = ((t & 1) << 2) | (t >> 1);            // swizzle of the 16-byte units of a Q row
+  const int ksw = ((t & 1) << 1) | ((t >> 1) << 3);     // swizzle of the columns of a K row
+  const double* qf0 = qscr + t * 32 + 2 * ((2 * g) ^ qsw);       // queries 4g, 4g+1
+  const double* qf1 = qscr + t * 32 + 2 * ((2 * g + 1) ^ qsw);   // queries 4g+2, 4g+3
+  const int kcol = 4 * (g >> 1) + (g & 1);
+  const double* kf0 = kscr + t * 16 + (kcol ^ ksw);              // key of tile column g, nt = 0
+  const double* kf1 = kscr + t * 16 + ((kcol + 2) ^ ksw);        // nt = 1
   fetch_q(0);
   ptx::tmem_wait_ld();
 #pragma unroll 1
@@ -229,16 +252,17 @@ __device__ __noinline__ void dot16(const __nv_bfloat16* __restrict__ krow, int64
     for (int e = 0; e < 8; ++e) {
       // a widened bf16 has a zero low word: only the high words are ever written, the low
       // words of the scratch were cleared when the kernel started
+      const int qpos = e * 32 + 2 * ((lane >> 1) ^ ((((e & 3) & 1) << 2) | ((e & 3) >> 1))) + (lane & 1);
       if constexpr (QHI) {
-        qhi[2 * (e * 32 + lane)] = qraw[e];
+        qhi[2 * qpos] = qraw[e];
       } else {
         const uint32_t wq = qraw[e >> 1];
-        qhi[2 * (e * 32 + lane)] = (uint32_t)__double2hiint((double)__uint_as_float((e & 1) ? (wq & 0xffff0000u) : (wq << 16)));
+        qhi[2 * qpos] = (uint32_t)__double2hiint((double)__uint_as_float((e & 1) ? (wq & 0xffff0000u) : (wq << 16)));
       }
       if (e < 4) {
         const uint32_t wk = (e >> 1) ? kraw.y : kraw.x;
-        khi[2 * ((4 * kh + e) * 16 + (lane & 15))] =
-            (uint32_t)__double2hiint((double)__uint_as_float((e & 1) ? (wk & 0xffff0000u) : (wk << 16)));
+        const int kpos = (4 * kh + e) * 16 + (key ^ (((e & 1) << 1) | ((e >> 1) << 3)));
+        khi[2 * kpos] = (uint32_t)__double2hiint((double)__uint_as_float((e & 1) ? (wk & 0xffff0000u) : (wk << 16)));
       }
     }
     const int kn = (k0 + 8) & (D - 1);      // next chunk's operands travel while this one is used
@@ -246,26 +270,27 @@ __device__ __noinline__ void dot16(const __nv_bfloat16* __restrict__ krow, int64
     fetch_q(kn);
     __syncwarp();
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      const double2 k01 = *reinterpret_cast<const double2*>(kscr + e * 16 + 4 * tp);
-      const double2 k23 = *reinterpret_cast<const double2*>(kscr + e * 16 + 4 * tp + 2);
-      const double2 q01 = *reinterpret_cast<const double2*>(qscr + e * 32 + 4 * qa);
-      const double2 q23 = *reinterpret_cast<const double2*>(qscr + e * 32 + 4 * qa + 2);
-      const double kd[4] = {k01.x, k01.y, k23.x, k23.y};
+    for (int ks = 0; ks < 2; ++ks) {
+      const double2 q01 = *reinterpret_cast<const double2*>(qf0 + ks * 128);
+      const double2 q23 = *reinterpret_cast<const double2*>(qf1 + ks * 128);
       const double qd[4] = {q01.x, q01.y, q23.x, q23.y};
+      const double kd[2] = {kf0[ks * 64], kf1[ks * 64]};
 #pragma unroll
-      for (int a = 0; a < 4; ++a)
+      for (int mt = 0; mt < 4; ++mt)
 #pragma unroll
-        for (int b = 0; b < 4; ++b) acc[a][b] = fma(kd[b], qd[a], acc[a][b]);
+        for (int nt = 0; nt < 2; ++nt) dmma_884(acc[mt][nt][0], acc[mt][nt][1], qd[mt], kd[nt]);
     }
     ptx::tmem_wait_ld();
     __syncwarp();
   }
   uint32_t yr[16];
 #pragma unroll
-  for (int a = 0; a < 4; ++a)
+  for (int mt = 0; mt < 4; ++mt)
 #pragma unroll
-    for (int b = 0; b < 4; ++b) yr[4 * a + b] = __float_as_uint(rne_e4m11(__dmul_rn(scale_d, acc[a][b])));
+    for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+      for (int e = 0; e < 2; ++e)
+        yr[4 * mt + 2 * nt + e] = __float_as_uint(rne_e4m11(__dmul_rn(scale_d, acc[mt][nt][e])));
   ptx::tmem_st16(tdst, yr);   // [query a][key b] of the lane's share, parked in its own TMEM lane
   ptx::tmem_wait_st();
 }
