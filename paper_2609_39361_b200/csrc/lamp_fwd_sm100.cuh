@@ -43,8 +43,8 @@ struct SmemLayout {
   static constexpr int kV = kKbf + kTK * kHalf * 2;               // 2 boxes [64 keys][64] bf16, SW128
   static constexpr int kPhi = kV + kTK * kHalf * 2;               // [128][64] bf16, SW128 K-major
   static constexpr int kPlo = kPhi + kBM * kTK * 2;
-  static constexpr int kLut = kPlo + kBM * kTK * 2;               // 128 x uint2
-  static constexpr int kDscr = kLut + 1024;                       // 4 groups x 384 doubles
+  static constexpr int kLut = kPlo + kBM * kTK * 2;               // 128 x uint4
+  static constexpr int kDscr = kLut + 2048;                       // 4 groups x 384 doubles
   static constexpr int kBar = kDscr + 4 * 384 * 8;                // mbarriers
   static constexpr int kMisc = kBar + 512;                        // tmem slot, lo masks
   static constexpr int kBytes = kMisc + 64;
@@ -387,6 +387,28 @@ __device__ __forceinline__ void unpack_e4m3x4(uint32_t w, float (&y)[4]) {
       : "=f"(y[0]), "=f"(y[1]), "=f"(y[2]), "=f"(y[3]) : "r"(w));
 }
 
+// The same as two packed f16 pairs (values 0, 1 and 2, 3), and a few packed-f16 helpers.
+__device__ __forceinline__ void unpack_e4m3x4_h2(uint32_t w, uint32_t& h01, uint32_t& h23) {
+  asm("{.reg .b16 lo, hi; mov.b32 {lo, hi}, %2; cvt.rn.f16x2.e4m3x2 %0, lo; cvt.rn.f16x2.e4m3x2 %1, hi;}"
+      : "=r"(h01), "=r"(h23) : "r"(w));
+}
+__device__ __forceinline__ uint32_t max_h2(uint32_t a, uint32_t b) {
+  uint32_t r;
+  asm("max.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+  return r;
+}
+__device__ __forceinline__ void h2_to_f32(uint32_t h, float& lo, float& hi) {
+  asm("{.reg .f16 l, u; mov.b32 {l, u}, %2; cvt.f32.f16 %0, l; cvt.f32.f16 %1, u;}" : "=f"(lo), "=f"(hi) : "r"(h));
+}
+// (m, m) - 0.5 * (y0, y1) in packed f16, then rounded to e4m3: the codes of the two shifts (low byte = value 0)
+__device__ __forceinline__ uint32_t half_shift_codes(uint32_t y2, uint32_t m2) {
+  uint32_t d;
+  unsigned short pk;
+  asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(y2), "r"(0xB800B800u), "r"(m2));
+  asm("cvt.rn.satfinite.e4m3x2.f16x2 %0, %1;" : "=h"(pk) : "r"(d));
+  return pk;
+}
+
 // e8 byte of an 8-bit exponential value (0xF8 = 1.0, E = 0 subnormals in units of 2^-33).
 __device__ __forceinline__ uint32_t enc_exp8(float e) {
   if (e == 0.0f) return 0u;
@@ -405,7 +427,7 @@ __device__ __forceinline__ uint32_t enc_exp8(float e) {
 template <int D, bool FULL, bool DUMP, int VAR>
 __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileGeom& g, const uint32_t (&yw)[16],
                                               const __nv_bfloat16* ktile, int64_t kstride, uint32_t tq,
-                                              const uint2* lut, double* dscr, unsigned char* phi, unsigned char* plo,
+                                              const uint4* lut, double* dscr, unsigned char* phi, unsigned char* plo,
                                               uint32_t tscratch, uint32_t& lo_dirty, RowState& st,
                                               float (&lam)[4], WarpCounters& wc, unsigned long long (&cks)[2],
                                               int dump_row0, int row0, long long* ph, uint64_t* pv_bar,
@@ -428,13 +450,27 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
 #pragma unroll
   for (int a = 0; a < 4; ++a) {
     float m = -INFINITY;
+    if (FULL) {
+      // all 16 keys visible: the maximum is taken on packed f16 pairs (every e4m3 value is an f16 value)
+      uint32_t h[8];
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      float y[4];
-      unpack_e4m3x4(yw[4 * a + c], y);
+      for (int c = 0; c < 4; ++c) unpack_e4m3x4_h2(yw[4 * a + c], h[2 * c], h[2 * c + 1]);
 #pragma unroll
-      for (int u = 0; u < 4; ++u)
-        if (vis<FULL>(g, 16 * th_own + 4 * c + u, 4 * qa + a)) m = fmaxf(m, y[u]);
+      for (int st = 4; st > 0; st >>= 1)
+#pragma unroll
+        for (int i = 0; i < st; ++i) h[i] = max_h2(h[i], h[i + st]);
+      float lo, hi;
+      h2_to_f32(h[0], lo, hi);
+      m = fmaxf(lo, hi);
+    } else {
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        float y[4];
+        unpack_e4m3x4(yw[4 * a + c], y);
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          if (vis<FULL>(g, 16 * th_own + 4 * c + u, 4 * qa + a)) m = fmaxf(m, y[u]);
+      }
     }
     cm[a] = m;
     wc.sat8 += m == 448.0f;
@@ -607,28 +643,30 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
 #pragma unroll
           for (int c = 0; c < 4; ++c) ya[c] = yw[4 * k + c];
         }
+      // half the truncated maximum, twice in a packed f16 pair: every e4m3 value, its half and the
+      // difference of two such halves (as far as its rounding to 4 significant bits goes: checked
+      // for all pairs of e4m3 values) are exact in f16, so the shift is formed on packed pairs
       const float m8h = 0.5f * trunc_e4m3(mh_sel);
+      uint32_t m2;
+      asm("cvt.rn.f16x2.f32 %0, %1, %1;" : "=r"(m2) : "f"(m8h));
       float s_hi = 0.0f, s_lo = 0.0f;
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
-        float y4[4];
-        unpack_e4m3x4(ya[c], y4);
+        uint32_t yh[2];
+        unpack_e4m3x4_h2(ya[c], yh[0], yh[1]);
 #pragma unroll
         for (int u = 0; u < 4; u += 2) {
           const int b = 4 * c + u;
           const bool ok0 = vis<FULL>(g, 16 * th_own + b, 4 * qa + a);
           const bool ok1 = vis<FULL>(g, 16 * th_own + b + 1, 4 * qa + a);
-          const float y0 = y4[u], y1 = y4[u + 1];
           float e0 = 0.0f, e1 = 0.0f;
           if (own8) {
-            // half the shift (exact), rounded to 4 significant bits by the conversion unit: its
-            // e4m3 code indexes the table (shifts below 2^-5 all map to 1.0, as in the 256-entry table)
-            unsigned short pk;
-            asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(pk)
-                : "f"(__fmaf_rn(y1, -0.5f, m8h)), "f"(__fmaf_rn(y0, -0.5f, m8h)));
-            const uint2 w0 = lut[pk & 0x7fu], w1 = lut[(pk >> 8) & 0x7fu];
-            if (ok0) { e0 = __uint_as_float(w0.x); s_lo += __uint_as_float(w0.y); s_hi += e0 - __uint_as_float(w0.y); }
-            if (ok1) { e1 = __uint_as_float(w1.x); s_lo += __uint_as_float(w1.y); s_hi += e1 - __uint_as_float(w1.y); }
+            // half the shift, rounded to 4 significant bits by the conversion unit: its e4m3 code
+            // indexes the table (shifts below 2^-5 all map to 1.0, as in the 256-entry table)
+            const uint32_t pk = half_shift_codes(yh[u >> 1], m2);
+            const uint4 w0 = lut[pk & 0x7fu], w1 = lut[(pk >> 8) & 0x7fu];
+            if (ok0) { e0 = __uint_as_float(w0.x); s_hi += __uint_as_float(w0.y); s_lo += __uint_as_float(w0.z); }
+            if (ok1) { e1 = __uint_as_float(w1.x); s_hi += __uint_as_float(w1.y); s_lo += __uint_as_float(w1.z); }
           }
           w[b >> 1] = pack_bf16(e0, e1);
           if (DUMP) {
@@ -850,7 +888,7 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
   unsigned char* vs = smem + L::kV;
   unsigned char* phi = smem + L::kPhi;
   unsigned char* plo = smem + L::kPlo;
-  uint2* lut = reinterpret_cast<uint2*>(smem + L::kLut);
+  uint4* lut = reinterpret_cast<uint4*>(smem + L::kLut);
   double* dscr_all = reinterpret_cast<double*>(smem + L::kDscr);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBar);
   uint32_t* tslot = reinterpret_cast<uint32_t*>(smem + L::kMisc);
@@ -894,7 +932,11 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
     ptx::tmem_relinquish();
     if (lane == 0) { ptx::prefetch_tensormap(&kmap); ptx::prefetch_tensormap(&vmap); }
   }
-  for (int i = tid; i < 128; i += kThreads) lut[i] = lut_g[i];
+  for (int i = tid; i < 128; i += kThreads) {
+    // value, its part of 2^-15 or more, its part below (the two partial sums of a row are exact in fp32)
+    const uint2 w = lut_g[i];
+    lut[i] = make_uint4(w.x, w.y ? 0u : w.x, w.y, 0u);
+  }
   for (int i = tid; i < 4 * 384; i += kThreads) dscr_all[i] = 0.0;
   {
     const __nv_bfloat16* qg = P.q + b * P.qs[0] + h * P.qs[1] + (int64_t)m0 * P.qs[2];
