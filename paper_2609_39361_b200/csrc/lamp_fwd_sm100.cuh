@@ -197,11 +197,12 @@ __device__ __forceinline__ void dmma_884(double& d0, double& d1, double a, doubl
 // the instruction's tiles so that a lane ends with exactly its own 4 queries x 4 keys: tile row
 // (mt, g) is query 4g + mt, tile column (nt, 2t + e) is key 4t + 2nt + e.
 // The fp32 -> fp64 conversions are slow on this GPU (they hold the scheduler for several cycles each),
-// so the warp converts each operand once per 8 channels into a small shared-memory scratch (16 keys
-// and 32 rows as doubles, columns swizzled by the channel so that the fragment loads of lanes with
-// different t fall into different banks) and every lane reads its fragments from there.
-// krow: global bf16 row of the sub-block's first key (lane l fetches key l % 16, channels
-// 4 (l / 16) .. +3 of every 8; the rows were just streamed through L2 by TMA).
+// so the warp converts each operand once into a small shared-memory scratch (two buffers of 4
+// channels: 16 keys and 32 rows as doubles, columns swizzled by the channel so that the fragment loads
+// of lanes with different t fall into different banks) and every lane reads its fragments from there;
+// the conversion of one step is issued behind the tensor-core instructions of the step before.
+// krow: global bf16 row of the sub-block's first key (lane l fetches key l % 16, 16 bytes per 8
+// channels; the rows were just streamed through L2 by TMA).
 // tq: TMEM columns holding the query row of this lane (row = lane of the group).  head_dim 128:
 // one column per channel, the high word of the channel as a double (the low word of a widened
 // bf16 is zero), converted once per CTA; head_dim 256: raw bf16, two channels per column, converted
@@ -213,19 +214,18 @@ __device__ __noinline__ void dot16(const __nv_bfloat16* __restrict__ krow, int64
   constexpr int QW = QHI ? 8 : 4;   // TMEM columns per 8 channels
   const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   __builtin_assume(__isShared(dscr));
-  double* kscr = dscr;          // [8 kk][16 keys]
-  double* qscr = dscr + 128;    // [8 kk][32 rows]
-  uint32_t* khi = reinterpret_cast<uint32_t*>(kscr) + 1;   // high words of the same
-  uint32_t* qhi = reinterpret_cast<uint32_t*>(qscr) + 1;
+  // two buffers of one 4-channel step each: [4 kk][16 keys] then [4 kk][32 rows]; while the tensor core
+  // works on one, the next step is converted into the other
+  uint32_t* hiw = reinterpret_cast<uint32_t*>(dscr) + 1;   // high words of the doubles
   double acc[4][2][2];          // [mt][nt][e]: query 4g + mt, key 4t + 2nt + e
 #pragma unroll
   for (int mt = 0; mt < 4; ++mt)
 #pragma unroll
     for (int nt = 0; nt < 2; ++nt) acc[mt][nt][0] = acc[mt][nt][1] = 0.0;
-  const int kh = lane >> 4;      // which four of a chunk's eight channels this lane converts for K
+  const int kh = lane >> 4;      // which two of a step's four channels this lane converts for K
   const int key = lane & 15;
-  const __nv_bfloat16* ksrc = krow + (int64_t)key * kstride + 4 * kh;
-  uint2 kraw = *reinterpret_cast<const uint2*>(ksrc);
+  const __nv_bfloat16* ksrc = krow + (int64_t)key * kstride;
+  uint4 kraw = *reinterpret_cast<const uint4*>(ksrc);
   uint32_t qraw[QW];
   auto fetch_q = [&](int k0) {
     if constexpr (QHI) {
@@ -236,51 +236,59 @@ __device__ __noinline__ void dot16(const __nv_bfloat16* __restrict__ krow, int64
       qraw[0] = v.x; qraw[1] = v.y; qraw[2] = v.z; qraw[3] = v.w;
     }
   };
-  // fragment addresses of this lane inside one 4-channel step (channel = 4 ks + t of the chunk)
+  // fragment addresses of this lane inside a buffer (its channel of the step is t)
   const int qsw = ((t & 1) << 2) | (t >> 1);            // swizzle of the 16-byte units of a Q row
   const int ksw = ((t & 1) << 1) | ((t >> 1) << 3);     // swizzle of the columns of a K row
-  const double* qf0 = qscr + t * 32 + 2 * ((2 * g) ^ qsw);       // queries 4g, 4g+1
-  const double* qf1 = qscr + t * 32 + 2 * ((2 * g + 1) ^ qsw);   // queries 4g+2, 4g+3
-  const int kcol = 4 * (g >> 1) + (g & 1);
-  const double* kf0 = kscr + t * 16 + (kcol ^ ksw);              // key of tile column g, nt = 0
-  const double* kf1 = kscr + t * 16 + ((kcol + 2) ^ ksw);        // nt = 1
+  const double* kf0 = dscr + t * 16 + ((4 * (g >> 1) + (g & 1)) ^ ksw);        // key of tile column g, nt = 0
+  const double* kf1 = dscr + t * 16 + ((4 * (g >> 1) + (g & 1) + 2) ^ ksw);    // nt = 1
+  const double* qf0 = dscr + 64 + t * 32 + 2 * ((2 * g) ^ qsw);                // queries 4g, 4g+1
+  const double* qf1 = dscr + 64 + t * 32 + 2 * ((2 * g + 1) ^ qsw);            // queries 4g+2, 4g+3
+  // convert step `half` (channels 4 half .. +3) of the fetched 8 channels into buffer `buf`.  A widened
+  // bf16 has a zero low word: only high words are written, the low words were cleared at kernel start
+  auto stage = [&](int half, int buf) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int qpos = buf * 192 + 64 + e * 32 + 2 * ((lane >> 1) ^ (((e & 1) << 2) | (e >> 1))) + (lane & 1);
+      if constexpr (QHI) {
+        hiw[2 * qpos] = qraw[4 * half + e];
+      } else {
+        const uint32_t wq = qraw[2 * half + (e >> 1)];
+        hiw[2 * qpos] = (uint32_t)__double2hiint((double)__uint_as_float((e & 1) ? (wq & 0xffff0000u) : (wq << 16)));
+      }
+    }
+    const uint32_t wk = half ? (kh ? kraw.w : kraw.z) : (kh ? kraw.y : kraw.x);   // channels 2kh, 2kh+1 of the step
+#pragma unroll
+    for (int e2 = 0; e2 < 2; ++e2) {
+      const int e = 2 * kh + e2;
+      const int kpos = buf * 192 + e * 16 + (key ^ (((e & 1) << 1) | ((e >> 1) << 3)));
+      hiw[2 * kpos] = (uint32_t)__double2hiint((double)__uint_as_float(e2 ? (wk & 0xffff0000u) : (wk << 16)));
+    }
+  };
+  auto step = [&](int buf) {
+    const double2 q01 = *reinterpret_cast<const double2*>(qf0 + buf * 192);
+    const double2 q23 = *reinterpret_cast<const double2*>(qf1 + buf * 192);
+    const double qd[4] = {q01.x, q01.y, q23.x, q23.y};
+    const double kd[2] = {kf0[buf * 192], kf1[buf * 192]};
+#pragma unroll
+    for (int mt = 0; mt < 4; ++mt)
+#pragma unroll
+      for (int nt = 0; nt < 2; ++nt) dmma_884(acc[mt][nt][0], acc[mt][nt][1], qd[mt], kd[nt]);
+  };
   fetch_q(0);
   ptx::tmem_wait_ld();
+  stage(0, 0);
+  __syncwarp();
 #pragma unroll 1
   for (int k0 = 0; k0 < D; k0 += 8) {
-#pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      // a widened bf16 has a zero low word: only the high words are ever written, the low
-      // words of the scratch were cleared when the kernel started
-      const int qpos = e * 32 + 2 * ((lane >> 1) ^ ((((e & 3) & 1) << 2) | ((e & 3) >> 1))) + (lane & 1);
-      if constexpr (QHI) {
-        qhi[2 * qpos] = qraw[e];
-      } else {
-        const uint32_t wq = qraw[e >> 1];
-        qhi[2 * qpos] = (uint32_t)__double2hiint((double)__uint_as_float((e & 1) ? (wq & 0xffff0000u) : (wq << 16)));
-      }
-      if (e < 4) {
-        const uint32_t wk = (e >> 1) ? kraw.y : kraw.x;
-        const int kpos = (4 * kh + e) * 16 + (key ^ (((e & 1) << 1) | ((e >> 1) << 3)));
-        khi[2 * kpos] = (uint32_t)__double2hiint((double)__uint_as_float((e & 1) ? (wk & 0xffff0000u) : (wk << 16)));
-      }
-    }
-    const int kn = (k0 + 8) & (D - 1);      // next chunk's operands travel while this one is used
-    kraw = *reinterpret_cast<const uint2*>(ksrc + kn);
+    step(0);
+    stage(1, 1);
+    const int kn = (k0 + 8) & (D - 1);      // the next 8 channels travel while these are used
+    kraw = *reinterpret_cast<const uint4*>(ksrc + kn);
     fetch_q(kn);
     __syncwarp();
-#pragma unroll
-    for (int ks = 0; ks < 2; ++ks) {
-      const double2 q01 = *reinterpret_cast<const double2*>(qf0 + ks * 128);
-      const double2 q23 = *reinterpret_cast<const double2*>(qf1 + ks * 128);
-      const double qd[4] = {q01.x, q01.y, q23.x, q23.y};
-      const double kd[2] = {kf0[ks * 64], kf1[ks * 64]};
-#pragma unroll
-      for (int mt = 0; mt < 4; ++mt)
-#pragma unroll
-        for (int nt = 0; nt < 2; ++nt) dmma_884(acc[mt][nt][0], acc[mt][nt][1], qd[mt], kd[nt]);
-    }
+    step(1);
     ptx::tmem_wait_ld();
+    stage(0, 0);
     __syncwarp();
   }
   uint32_t yr[16];
