@@ -181,6 +181,13 @@ int lamp_attn_fwd_digest(const void* q, const void* k, const void* v, void* out,
  * Inputs must be finite with |x| < 2^100.  Asynchronous on the stream. */
 int lamp_attn_debug_round_e4m3(const float* in, float* out, size_t n, void* cuda_stream);
 
+/* Test hook: the kernel's 16-bit exponential (Sec. 3.3: exp of the shifted logit, correctly rounded to
+ * ue5m11 = 12 significant bits with the quantum 2^-41 below 2^-30) applied to n fp32 values.
+ *   in, out  device, n floats each (may alias)
+ * The kernel only ever passes arguments with at most 12 significant bits; the tests sweep that whole
+ * domain against the correctly rounded result.  Asynchronous on the stream. */
+int lamp_attn_debug_exp16(const float* in, float* out, size_t n, void* cuda_stream);
+
 /* Wait for the stream, then copy the counters of the last lamp_attn_fwd on the current
  * device to *host_out.  Returns LAMP_ERR_DEVICE_TIMEOUT if that kernel gave up a wait. */
 int lamp_attn_get_stats(lamp_attn_stats* host_out, void* cuda_stream);

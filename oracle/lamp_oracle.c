@@ -182,6 +182,10 @@ float lamp_oracle_exp16(float a) {
   return (float)r;   /* 12 significant bits: exact in fp32 unless it overflows to inf */
 }
 
+void lamp_oracle_exp16_array(const float* in, float* out, size_t n) {
+  for (size_t i = 0; i < n; ++i) out[i] = lamp_oracle_exp16(in[i]);
+}
+
 /* --------------------------------------------------------- stage 2 (eq. 8) */
 
 /* xi[theta][j]: per sub-block, per query sum of (omega_hat - e) e  (0 for sub-blocks

@@ -79,6 +79,8 @@ def lib():
         L.lamp_oracle_chain16.argtypes = [C.c_void_p, C.c_void_p, C.c_int]
         L.lamp_oracle_chain8.restype = f32
         L.lamp_oracle_chain8.argtypes = [C.c_void_p, C.c_void_p, C.c_int]
+        L.lamp_oracle_exp16_array.restype = None
+        L.lamp_oracle_exp16_array.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t]
         L.lamp_oracle_rne_e4m3_array.restype = None
         L.lamp_oracle_rne_e4m3_array.argtypes = [C.c_void_p, C.c_void_p, C.c_int64]
         L.lamp_oracle_units.restype = C.c_int
@@ -92,6 +94,14 @@ def rne_e4m3_array(x: np.ndarray) -> np.ndarray:
     x = np.ascontiguousarray(x, np.float32)
     out = np.empty_like(x)
     lib().lamp_oracle_rne_e4m3_array(x.ctypes.data_as(C.c_void_p), out.ctypes.data_as(C.c_void_p), x.size)
+    return out
+
+
+def exp16_array(x: np.ndarray) -> np.ndarray:
+    """The oracle's 16-bit exponential, element by element, on a float32 array."""
+    x = np.ascontiguousarray(x, np.float32)
+    out = np.empty_like(x)
+    lib().lamp_oracle_exp16_array(x.ctypes.data_as(C.c_void_p), out.ctypes.data_as(C.c_void_p), x.size)
     return out
 
 

@@ -10,7 +10,7 @@ _LIB_PATH = os.path.join(_HERE, "liblamp_attn.so")
 LAMP_FORCE_16BIT, LAMP_FORCE_8BIT, LAMP_NO_STAGE1, LAMP_OUT_FP32, LAMP_COMPACT_BRANCH, LAMP_H16_SEQ, LAMP_SR_E4M3 = 1, 2, 4, 8, 16, 32, 64
 
 EXPORTS = ("lamp_attn_default_params", "lamp_attn_contiguous_strides", "lamp_attn_workspace_bytes",
-           "lamp_attn_fwd", "lamp_attn_fwd_digest", "lamp_attn_debug_round_e4m3", "lamp_attn_get_stats", "lamp_attn_last_cuda_error", "lamp_attn_strerror")
+           "lamp_attn_fwd", "lamp_attn_fwd_digest", "lamp_attn_debug_round_e4m3", "lamp_attn_debug_exp16", "lamp_attn_get_stats", "lamp_attn_last_cuda_error", "lamp_attn_strerror")
 
 
 class LampAttnError(RuntimeError):
@@ -66,6 +66,8 @@ def library():
         L.lamp_attn_fwd_digest.argtypes = [C.c_void_p] * 6 + [PP, C.c_void_p, C.c_void_p]
         L.lamp_attn_debug_round_e4m3.restype = C.c_int
         L.lamp_attn_debug_round_e4m3.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.lamp_attn_debug_exp16.restype = C.c_int
+        L.lamp_attn_debug_exp16.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         L.lamp_attn_get_stats.restype = C.c_int
         L.lamp_attn_get_stats.argtypes = [C.POINTER(LampAttnStats), C.c_void_p]
         L.lamp_attn_last_cuda_error.restype = C.c_int; L.lamp_attn_last_cuda_error.argtypes = []
@@ -124,6 +126,16 @@ def lamp_attn_debug_round_e4m3(x, out=None, stream=None):
     s = torch.cuda.current_stream().cuda_stream if stream is None else stream
     _check(library().lamp_attn_debug_round_e4m3(_ptr(x), _ptr(out), x.numel(), C.c_void_p(s)),
            "lamp_attn_debug_round_e4m3")
+    return out
+
+
+def lamp_attn_debug_exp16(x, out=None, stream=None):
+    """The kernel's 16-bit exponential applied to a CUDA fp32 tensor (test hook)."""
+    import torch
+    assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous()
+    out = torch.empty_like(x) if out is None else out
+    s = torch.cuda.current_stream().cuda_stream if stream is None else stream
+    _check(library().lamp_attn_debug_exp16(_ptr(x), _ptr(out), x.numel(), C.c_void_p(s)), "lamp_attn_debug_exp16")
     return out
 
 

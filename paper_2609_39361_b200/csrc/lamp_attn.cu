@@ -276,6 +276,11 @@ __global__ void lamp_round_e4m3_kernel(const float* __restrict__ in, float* __re
   }
 }
 
+__global__ void lamp_exp16_kernel(const float* __restrict__ in, float* __restrict__ out, size_t n) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+    out[i] = exp16(in[i]);
+}
+
 // Scratch of the digest call: two 64-bit checksums per (group, key tile) pair.  Device code may
 // name the array; host code may not use the name as a pointer (on the host it is only a handle
 // for cudaGetSymbolAddress).
@@ -346,6 +351,19 @@ int lamp_attn_debug_round_e4m3(const float* in, float* out, size_t n, void* cuda
   const size_t pairs = (n + 1) / 2;
   const int blocks = (int)(pairs / 256 + 1 < 4096 ? pairs / 256 + 1 : 4096);
   lamp_round_e4m3_kernel<<<blocks, 256, 0, (cudaStream_t)cuda_stream>>>(in, out, n);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  return LAMP_OK;
+}
+
+int lamp_attn_debug_exp16(const float* in, float* out, size_t n, void* cuda_stream) {
+  if (!in || !out) return LAMP_ERR_INVALID_ARG;
+  int dev = 0;
+  int rc = ensure_device(&dev);
+  if (rc) return rc;
+  if (n == 0) return LAMP_OK;
+  const int blocks = (int)(n / 256 + 1 < 4096 ? n / 256 + 1 : 4096);
+  lamp_exp16_kernel<<<blocks, 256, 0, (cudaStream_t)cuda_stream>>>(in, out, n);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
   return LAMP_OK;

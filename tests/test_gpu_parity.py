@@ -27,6 +27,25 @@ def test_rounding_of_the_chain_against_the_oracle_in_bulk():
     assert np.array_equal(np.signbit(got[nz]), np.signbit(want[nz]))
 
 
+def test_sixteen_bit_exponential_on_its_whole_domain():
+    """The kernel only ever exponentiates shifts with at most 12 significant bits.  Every such value from
+    -50 to 89 (all 2^11 mantissas of every binade down to 2^-40, both signs, and zero), plus the ranges
+    that round to 0 and overflow: the kernel's evaluation (fp64 exponential, then one rounding) gives the
+    oracle's correctly rounded result bit for bit."""
+    import paper_2609_39361_b200 as lamp
+    mant = np.arange(1 << 11, dtype=np.uint32) << 12                       # 11 fraction bits
+    exps = np.arange(127 - 40, 127 + 7, dtype=np.uint32)                   # 2^-40 .. 2^6
+    bits = ((exps[:, None] << 23) | mant[None, :]).reshape(-1)
+    x = np.concatenate([bits.view(np.float32), (bits | 0x80000000).view(np.float32),
+                        np.array([0.0, -0.0, -50.0, -50.03125, -60.0, -700.0, -1e30, 89.0, 89.0625, 100.0, 1e30],
+                                 np.float32)])
+    x = x[(x <= 1e30)]
+    got = lamp.lamp_attn_debug_exp16(torch.from_numpy(x).cuda()).cpu().numpy()
+    want = oracle.exp16_array(x)
+    bad = np.flatnonzero(~((got == want) | (np.isinf(got) & np.isinf(want))))
+    assert bad.size == 0, (x[bad][:8], got[bad][:8], want[bad][:8])
+
+
 def test_config0_dense():
     cfg = li.CONFIGS[0]
     q, k, v = li.make_qkv(cfg)
