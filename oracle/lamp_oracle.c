@@ -266,6 +266,7 @@ static double exact_rowsum(const float Ef[TK][BQ], int j, int* big) {
 }
 
 static int pair_valid(const lamp_oracle_params* p, int64_t i, int64_t j) {
+  if (i >= p->seqlen || j >= p->seqlen) return 0;   /* the last group / tile of a ragged sequence */
   if (p->causal && i > j) return 0;
   if (p->window > 0 && j - i >= p->window) return 0;
   return 1;
@@ -273,7 +274,7 @@ static int pair_valid(const lamp_oracle_params* p, int64_t i, int64_t j) {
 
 /* One unit = (batch b, query head h, group g of 32 query rows): Algorithm 1's
  * per-warp body over all key tiles in ascending order.
- * out [32][D], lse [32], flags [N/64], checks [N/64][2] (or NULL),
+ * out [32][D], lse [32], flags [ceil(N/64)], checks [ceil(N/64)][2] (or NULL),
  * y8 / e8 [32][N] bytes (or NULL).                                              */
 static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
                         const lamp_oracle_params* p, int b, int h, int g, float* out,
@@ -284,7 +285,7 @@ static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
   const uint16_t* Q = q + ((int64_t)(b * p->heads_q + h) * N + (int64_t)g * BQ) * D;
   const uint16_t* K = k + (int64_t)(b * p->heads_kv + hk) * N * D;
   const uint16_t* V = v + (int64_t)(b * p->heads_kv + hk) * N * D;
-  const int ntiles = N / TK;
+  const int ntiles = (N + TK - 1) / TK;
   const int64_t j0 = (int64_t)g * BQ;
 
   float* qs = (float*)malloc(sizeof(float) * BQ * D);
@@ -293,7 +294,7 @@ static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
   for (int j = 0; j < BQ; ++j) {
     mu[j] = -INFINITY;
     omega[j] = 0.0f;
-    for (int c = 0; c < D; ++c) qs[j * D + c] = bf16_to_float(Q[j * D + c]) * p->scale;
+    for (int c = 0; c < D; ++c) qs[j * D + c] = j0 + j < N ? bf16_to_float(Q[j * D + c]) * p->scale : 0.0f;
   }
   if (y8d) memset(y8d, 0x7F, (size_t)BQ * N);
   if (e8d) memset(e8d, 0xFF, (size_t)BQ * N);
@@ -317,6 +318,7 @@ static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
     for (int i = 0; i < TK; ++i)
       for (int j = 0; j < BQ; ++j) {
         float c = 0.0f;
+        if (!val[i][j]) { Y8[i][j] = 0.0f; continue; }   /* never used, and may lie past the tensors */
         for (int kk = 0; kk < D; ++kk)
           {
             float tkk = fmaf(bf16_to_float(K[(i0 + i) * D + kk]), qs[j * D + kk], c);
@@ -494,6 +496,11 @@ static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
   }
 
   for (int j = 0; j < BQ; ++j) {
+    if (j0 + j >= N) {   /* rows past the end of a ragged sequence */
+      for (int c = 0; c < D; ++c) out[j * D + c] = 0.0f;
+      lse[j] = 0.0f;
+      continue;
+    }
     for (int c = 0; c < D; ++c) out[j * D + c] = (float)(O[j * D + c] / (double)omega[j]);
     lse[j] = (float)((double)mu[j] + log((double)omega[j]));
   }
@@ -511,17 +518,19 @@ static void stats_add(lamp_oracle_stats* a, const lamp_oracle_stats* b) {
 
 /* Run the listed units.  q, k, v: host, bf16 bit patterns, contiguous
  * [B, H, N, D].  units: n_units triples (b, h, g).  Outputs are per unit:
- * out [n][32][D] fp32, lse [n][32], flags [n][N/64] (bits 0-3 stage-1 set,
- * bits 4-7 stage-2 set), checks [n][N/64][2] or NULL, y8 / e8 [n][32][N] or NULL.
+ * out [n][32][D] fp32, lse [n][32], flags [n][ceil(N/64)] (bits 0-3 stage-1 set,
+ * bits 4-7 stage-2 set), checks [n][ceil(N/64)][2] or NULL, y8 / e8 [n][32][N] or NULL.
+ * N need not be a multiple of the tile sizes: rows and keys past N do not exist (rows past N of the
+ * last group come back as zeros).
  * Returns 0, or -1 on an unsupported shape. */
 int lamp_oracle_units(const uint16_t* q, const uint16_t* k, const uint16_t* v,
                       const lamp_oracle_params* p, int64_t n_units, const int32_t* units,
                       float* out, float* lse, uint8_t* flags, uint64_t* checks, uint8_t* y8,
                       uint8_t* e8, lamp_oracle_stats* stats) {
-  if (p->seqlen % TK || p->seqlen % BQ || p->heads_q % p->heads_kv || p->head_dim <= 0 ||
+  if (p->seqlen <= 0 || p->heads_q % p->heads_kv || p->head_dim <= 0 || p->head_dim > 256 ||
       p->delta < 0.0f || (p->window > 0 && !p->causal))
     return -1;
-  const int N = p->seqlen, D = p->head_dim, nt = N / TK;
+  const int N = p->seqlen, D = p->head_dim, nt = (N + TK - 1) / TK;
   lamp_oracle_stats total;
   memset(&total, 0, sizeof(total));
   for (int i = 0; i < 256; ++i) g_lut8[i] = lamp_oracle_lut8((uint8_t)i);

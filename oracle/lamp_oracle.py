@@ -140,8 +140,8 @@ def run_units(q, k, v, units, *, causal=True, window=0, scale=None, tau=0.5, del
     p = Params(B, Hq, Hkv, N, D, int(causal), int(window), float(scale), float(tau), float(delta), int(flags), int(sr_seed))
     out = np.zeros((n, 32, D), np.float32)
     lse = np.zeros((n, 32), np.float32)
-    fl = np.zeros((n, N // 64), np.uint8)
-    ck = np.zeros((n, N // 64, 2), np.uint64) if checksums else None
+    fl = np.zeros((n, (N + 63) // 64), np.uint8)
+    ck = np.zeros((n, (N + 63) // 64, 2), np.uint64) if checksums else None
     y8 = np.zeros((n, 32, N), np.uint8) if dumps else None
     e8 = np.zeros((n, 32, N), np.uint8) if dumps else None
     st = Stats()
@@ -154,7 +154,7 @@ def run_units(q, k, v, units, *, causal=True, window=0, scale=None, tau=0.5, del
 
 
 def all_units(B, Hq, N):
-    g = np.stack(np.meshgrid(np.arange(B), np.arange(Hq), np.arange(N // 32), indexing="ij"), -1)
+    g = np.stack(np.meshgrid(np.arange(B), np.arange(Hq), np.arange((N + 31) // 32), indexing="ij"), -1)
     return g.reshape(-1, 3).astype(np.int32)
 
 

@@ -398,6 +398,37 @@ def test_compact_layout_branch(small):
     assert comp.stats["stage1_flagged"] + comp.stats["stage2_flagged"] > plain.stats["stage1_flagged"] + plain.stats["stage2_flagged"]
 
 
+def test_ragged_sequence_lengths():
+    """N need not be a multiple of the tile sizes.  Causal attention on a prefix is a prefix of causal
+    attention: every complete group of 32 rows agrees bit for bit with the run on the longer sequence; the
+    last, partial group still has rows that sum to one and, with everything in 16 bits, matches fp64
+    attention (causal and not) within the 16-bit bound."""
+    cfg = li.CONFIGS[1]
+    q, k, v = li.make_qkv(cfg, Hq=2, Hkv=1, N=256, seed=9)
+    sc = li.softmax_scale(128)
+    full = oracle.run_all(q, k, v, scale=sc)
+    for N in (200, 161, 97):
+        qn, kn, vn = q[:, :, :N].contiguous(), k[:, :, :N].contiguous(), v[:, :, :N].contiguous()
+        r = oracle.run_all(qn, kn, vn, scale=sc)
+        G, T = (N + 31) // 32, (N + 63) // 64
+        assert r.flags.shape == (2 * G, T)
+        for u, (b, h, g) in enumerate(r.units):
+            uf = h * 8 + g
+            if 32 * g + 32 <= N:
+                assert np.array_equal(r.out[u], full.out[uf]) and np.array_equal(r.lse[u], full.lse[uf])
+                assert np.array_equal(r.flags[u], full.flags[uf, :T])
+            else:
+                assert np.all(r.out[u][N - 32 * g:] == 0)
+        ones = oracle.run_all(qn, kn, torch.ones_like(vn), scale=sc)
+        valid = np.concatenate([np.arange(32) + 32 * g < N for _ in range(2) for g in range(G)])
+        assert np.abs(ones.out.reshape(-1, 128)[valid] - 1.0).max() < 1e-6
+        for causal in (True, False):
+            r16 = oracle.run_all(qn, kn, vn, scale=sc, causal=causal, flags=oracle.FORCE_16BIT)
+            o, l, _ = ref_attention(qn, kn, vn, sc, causal=causal)
+            got = torch.from_numpy(r16.out).reshape(1, 2, G * 32, 128)[:, :, :N].double()
+            assert (got - o).abs().max() < 0.1 and (got - o).norm() / o.norm() < 5e-3
+
+
 def test_rows_sum_to_one_and_units_are_independent(small):
     q, k, v, sc = small
     ones = torch.ones_like(v)
