@@ -70,7 +70,8 @@ typedef enum lamp_attn_error {
 
 typedef struct lamp_attn_params {
   int32_t batch, heads_q, heads_kv; /* heads_q % heads_kv == 0 (grouped-query attention)      */
-  int32_t seqlen;                   /* multiple of 128                                         */
+  int32_t seqlen;                   /* any length >= 1; rows and keys past it do not exist.  In the
+                                       shapes below seqlen/32 and seqlen/64 are rounded up        */
   int32_t head_dim;                 /* 128 or 256                                              */
   int64_t q_strides[3], k_strides[3], v_strides[3], o_strides[3];
   int32_t causal;                   /* 0 / 1                                                   */

@@ -185,14 +185,14 @@ def forward(q, k, v, *, causal=True, window=0, scale=None, threshold=0.5, delta=
     p.sr_seed = int(sr_seed)
     res = {"out": out}
     lse = torch.empty(B, Hq, N, device=q.device, dtype=torch.float32) if want_lse else None
-    fm = torch.empty(B, Hq, N // 32, N // 64, device=q.device, dtype=torch.uint8) if want_flags else None
+    fm = torch.empty(B, Hq, (N + 31) // 32, (N + 63) // 64, device=q.device, dtype=torch.uint8) if want_flags else None
     if dump is not None:
         p.dbg_batch, p.dbg_head = dump
         res["y8"] = torch.full((N, N), 0x7F, device=q.device, dtype=torch.uint8)
         res["e8"] = torch.full((N, N), 0xFF, device=q.device, dtype=torch.uint8)
         p.dbg_y8, p.dbg_e8 = res["y8"].data_ptr(), res["e8"].data_ptr()
     if checksums:
-        res["checks"] = torch.empty(B, Hq, N // 32, N // 64, 2, device=q.device, dtype=torch.int64)
+        res["checks"] = torch.empty(B, Hq, (N + 31) // 32, (N + 63) // 64, 2, device=q.device, dtype=torch.int64)
         p.dbg_checksums = res["checks"].data_ptr()
     ws_bytes = lamp_attn_workspace_bytes(p)
     ws = torch.empty(ws_bytes, device=q.device, dtype=torch.uint8) if ws_bytes else None

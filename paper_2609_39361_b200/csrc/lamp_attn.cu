@@ -177,7 +177,6 @@ static int check_params(const void* q, const void* k, const void* v, void* out,
       (p->dbg_batch < 0 || p->dbg_batch >= p->batch || p->dbg_head < 0 || p->dbg_head >= p->heads_q))
     return LAMP_ERR_INVALID_ARG;
   if (p->head_dim != 128 && p->head_dim != 256) return LAMP_ERR_UNSUPPORTED_SHAPE;
-  if (p->seqlen % kBM) return LAMP_ERR_UNSUPPORTED_SHAPE;
   if (p->batch > 65535 || p->heads_q > 65535) return LAMP_ERR_UNSUPPORTED_SHAPE;
   const int D = p->head_dim;
   if (!strides_ok(p->q_strides, D) || !strides_ok(p->k_strides, D) ||
@@ -218,7 +217,7 @@ int lamp_attn_fwd(const void* q, const void* k, const void* v, void* out, float*
   e = cudaMemsetAsync(stats_ptr, 0, sizeof(DeviceStats), stream);
   if (e != cudaSuccess) return cuda_fail(e);
 
-  const size_t ngt = (size_t)p->batch * p->heads_q * (p->seqlen / kBQ) * (p->seqlen / kTK);
+  const size_t ngt = (size_t)p->batch * p->heads_q * ((p->seqlen + kBQ - 1) / kBQ) * ((p->seqlen + kTK - 1) / kTK);
   if (flag_mask) {
     e = cudaMemsetAsync(flag_mask, 0, ngt, stream);
     if (e != cudaSuccess) return cuda_fail(e);
@@ -236,7 +235,7 @@ int lamp_attn_fwd(const void* q, const void* k, const void* v, void* out, float*
   rc = make_kv_map(&vmap, v, p->v_strides, p->head_dim, p->seqlen, p->heads_kv, p->batch);
   if (rc) return rc;
   const bool dump = p->dbg_y8 || p->dbg_e8 || p->dbg_checksums;
-  dim3 grid(p->seqlen / kBM, p->heads_q, p->batch), block(kThreads);
+  dim3 grid((p->seqlen + kBM - 1) / kBM, p->heads_q, p->batch), block(kThreads);
   const uint2* lutp = (const uint2*)lut_ptr;
   DeviceStats* dsp = (DeviceStats*)stats_ptr;
 #define LAMP_LAUNCH(D_, DUMP_, VAR_) \
@@ -313,9 +312,9 @@ int lamp_attn_fwd_digest(const void* q, const void* k, const void* v, void* out,
                          uint8_t* flag_mask, const lamp_attn_params* p, uint64_t* digest,
                          void* cuda_stream) {
   if (!p || !digest) return LAMP_ERR_INVALID_ARG;
-  if (p->batch <= 0 || p->heads_q <= 0 || p->seqlen <= 0 || p->seqlen % kBM) return LAMP_ERR_INVALID_ARG;
+  if (p->batch <= 0 || p->heads_q <= 0 || p->seqlen <= 0) return LAMP_ERR_INVALID_ARG;
   const unsigned long long n_pairs =
-      (unsigned long long)p->batch * p->heads_q * (p->seqlen / kBQ) * (p->seqlen / kTK);
+      (unsigned long long)p->batch * p->heads_q * ((p->seqlen + kBQ - 1) / kBQ) * ((p->seqlen + kTK - 1) / kTK);
   if (n_pairs > LAMP_DIGEST_MAX_PAIRS) return LAMP_ERR_UNSUPPORTED_SHAPE;   // beyond the built-in scratch
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);

@@ -66,11 +66,11 @@ enum Bar {
 };
 
 struct TileGeom {
-  int i0, j0, causal, window;
+  int i0, j0, causal, window, n;   // n: sequence length (rows and keys past it do not exist)
 };
 template <bool FULL>
 __device__ __forceinline__ bool vis(const TileGeom& g, int i, int j) {
-  return FULL || pair_valid(g.causal, g.window, g.i0 + i, g.j0 + j);
+  return FULL || (g.i0 + i < g.n && g.j0 + j < g.n && pair_valid(g.causal, g.window, g.i0 + i, g.j0 + j));
 }
 
 __device__ __forceinline__ void fma_x2(float& d0, float& d1, float a0, float a1, uint64_t bb, float c0, float c1) {
@@ -208,7 +208,7 @@ __device__ __forceinline__ void dmma_884(double& d0, double& d1, double a, doubl
 // bf16 is zero), converted once per CTA; head_dim 256: raw bf16, two channels per column, converted
 // here.  dscr: 384 doubles for the warp.
 template <int D>
-__device__ __noinline__ void dot16(const __nv_bfloat16* __restrict__ krow, int64_t kstride, uint32_t tq,
+__device__ __noinline__ void dot16(const __nv_bfloat16* __restrict__ krow, int64_t kstride, int nkey, uint32_t tq,
                                    double* dscr, double scale_d, uint32_t tdst) {
   constexpr bool QHI = (D == 128);
   constexpr int QW = QHI ? 8 : 4;   // TMEM columns per 8 channels
@@ -224,7 +224,7 @@ __device__ __noinline__ void dot16(const __nv_bfloat16* __restrict__ krow, int64
     for (int nt = 0; nt < 2; ++nt) acc[mt][nt][0] = acc[mt][nt][1] = 0.0;
   const int kh = lane >> 4;      // which two of a step's four channels this lane converts for K
   const int key = lane & 15;
-  const __nv_bfloat16* ksrc = krow + (int64_t)key * kstride;
+  const __nv_bfloat16* ksrc = krow + (int64_t)min(key, nkey - 1) * kstride;   // nkey: keys that exist (< 16 at the ragged end)
   uint4 kraw = *reinterpret_cast<const uint4*>(ksrc);
   uint32_t qraw[QW];
   auto fetch_q = [&](int k0) {
@@ -309,7 +309,7 @@ __device__ __noinline__ void dot16(const __nv_bfloat16* __restrict__ krow, int64
 // q_quad: the lane's quad in the shared-memory Q operand of the chain (fp32 q*scale for head_dim 128,
 // raw bf16 q for 256); K rows from global memory, 16 bytes (8 channels) per key at a time.
 template <int D>
-__device__ __noinline__ void dot16_seq(const __nv_bfloat16* __restrict__ krow, int64_t kstride,
+__device__ __noinline__ void dot16_seq(const __nv_bfloat16* __restrict__ krow, int64_t kstride, int nkey,
                                        const unsigned char* q_quad, float scale, uint32_t tdst) {
   constexpr bool QF32 = (D == 128);
   const int tp = threadIdx.x & 3;
@@ -321,7 +321,7 @@ __device__ __noinline__ void dot16_seq(const __nv_bfloat16* __restrict__ krow, i
   const __nv_bfloat16* ksrc = krow + (int64_t)(4 * tp) * kstride;
   uint4 kraw[4];
 #pragma unroll
-  for (int b = 0; b < 4; ++b) kraw[b] = *reinterpret_cast<const uint4*>(ksrc + b * kstride);
+  for (int b = 0; b < 4; ++b) kraw[b] = *reinterpret_cast<const uint4*>(krow + (int64_t)min(4 * tp + b, nkey - 1) * kstride);
 #pragma unroll 1
   for (int k0 = 0; k0 < D; k0 += 8) {
     uint4 cur[4];
@@ -329,7 +329,7 @@ __device__ __noinline__ void dot16_seq(const __nv_bfloat16* __restrict__ krow, i
     for (int b = 0; b < 4; ++b) cur[b] = kraw[b];
     const int kn = (k0 + 8) & (D - 1);
 #pragma unroll
-    for (int b = 0; b < 4; ++b) kraw[b] = *reinterpret_cast<const uint4*>(ksrc + b * kstride + kn);
+    for (int b = 0; b < 4; ++b) kraw[b] = *reinterpret_cast<const uint4*>(krow + (int64_t)min(4 * tp + b, nkey - 1) * kstride + kn);
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
       float q4[4];
@@ -448,8 +448,9 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
   const bool skip1 = (P.flags & (LAMP_FORCE_8BIT | LAMP_NO_STAGE1)) != 0;
   auto logits16 = [&](int th) {
     const __nv_bfloat16* kr = ktile + (int64_t)(16 * th) * kstride;
-    if constexpr (VAR == 1) dot16_seq<D>(kr, kstride, q_quad, P.scale, tscratch + 16 * th);
-    else dot16<D>(kr, kstride, tq, dscr, scale_d, tscratch + 16 * th);
+    const int nkey = min(16, g.n - (g.i0 + 16 * th));
+    if constexpr (VAR == 1) dot16_seq<D>(kr, kstride, nkey, q_quad, P.scale, tscratch + 16 * th);
+    else dot16<D>(kr, kstride, nkey, tq, dscr, scale_d, tscratch + 16 * th);
   };
 
   // ---- per sub-block, per query maxima; which sub-blocks are active --------------------------
@@ -489,7 +490,7 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
     bool act = true;
     if (!FULL) {
       const int s0 = g.i0 + 16 * th;
-      act = (!g.causal || s0 <= g.j0 + 31) && (g.window == 0 || g.j0 - (s0 + 15) < g.window);
+      act = s0 < g.n && (!g.causal || s0 <= min(g.j0 + 31, g.n - 1)) && (g.window == 0 || g.j0 - (s0 + 15) < g.window);
     }
     actmask |= (uint32_t)act << th;
   }
@@ -904,14 +905,14 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
   int* status = &gstats->status;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int ntq = P.seqlen / kBM;
+  const int ntq = (P.seqlen + kBM - 1) / kBM;
   const int qt = ntq - 1 - (int)blockIdx.x;   // long (late) query tiles first
   const int h = blockIdx.y, b = blockIdx.z;
   const int hk = h / (P.heads_q / P.heads_kv);
   const int m0 = qt * kBM;
 
-  int t_begin = 0, t_end = P.seqlen / kTK;
-  if (P.causal) t_end = min(t_end, (m0 + kBM - 1) / kTK + 1);
+  int t_begin = 0, t_end = (P.seqlen + kTK - 1) / kTK;
+  if (P.causal) t_end = min(t_end, (min(m0 + kBM, P.seqlen) - 1) / kTK + 1);
   if (P.window > 0) t_begin = max(0, m0 - P.window + 1) / kTK;
   const int T = t_end - t_begin;
   const int M = T * NH;                       // half-tiles of the K (and V) stream
@@ -950,7 +951,8 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
     const __nv_bfloat16* qg = P.q + b * P.qs[0] + h * P.qs[1] + (int64_t)m0 * P.qs[2];
     for (int c = tid; c < kBM * D / 8; c += kThreads) {
       const int row = c % kBM, k0 = (c / kBM) * 8;   // consecutive threads -> consecutive rows
-      const uint4 raw = *reinterpret_cast<const uint4*>(qg + (int64_t)row * P.qs[2] + k0);
+      const int rsrc = min(row, P.seqlen - 1 - m0);  // rows past the end of the sequence repeat the last one (never used)
+      const uint4 raw = *reinterpret_cast<const uint4*>(qg + (int64_t)rsrc * P.qs[2] + k0);
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
         const uint32_t w = (&raw.x)[e >> 1];
@@ -1095,7 +1097,8 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
     bool ok = true;
     for (int n = side; n < T && ok; n += 2) {
       const int i0 = (t_begin + n) * kTK;
-      const bool any = (!P.causal || i0 <= j0 + 31) && (P.window == 0 || j0 - (i0 + 63) < P.window);
+      const bool any = j0 < P.seqlen && (!P.causal || i0 <= min(j0 + 31, P.seqlen - 1)) &&
+                       (P.window == 0 || j0 - (i0 + 63) < P.window);
       float acc[4][16];
 #pragma unroll
       for (int hh = 0; hh < NH; ++hh) {
@@ -1145,7 +1148,7 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
     const int grp = warp;
     const int qa = lane >> 2;
     const int j0 = m0 + grp * kBQ;
-    const int ntk = P.seqlen / kTK;
+    const int ntk = (P.seqlen + kTK - 1) / kTK;
     const bool dump_rows = DUMP && b == P.dbg_batch && h == P.dbg_head;
     const __nv_bfloat16* kg = P.k + b * P.ks[0] + hk * P.ks[1];
     double* dscr = dscr_all + grp * 384;
@@ -1153,7 +1156,7 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
     const uint32_t tlane = tbase + ((uint32_t)(grp * 32) << 16);
     const uint32_t tscr = tlane + kColScr, tq = tlane + kColQ, tring = tlane + kColRing;
     {
-      const __nv_bfloat16* qrow = P.q + b * P.qs[0] + h * P.qs[1] + (int64_t)(j0 + lane) * P.qs[2];
+      const __nv_bfloat16* qrow = P.q + b * P.qs[0] + h * P.qs[1] + (int64_t)min(j0 + lane, P.seqlen - 1) * P.qs[2];
 #pragma unroll 1
       for (int c0 = 0; c0 < 128; c0 += 16) {
         uint32_t r[16];
@@ -1188,9 +1191,11 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
     for (int n = 0; n < T && ok; ++n) {
       const int t = t_begin + n, i0 = t * kTK;
       TileGeom g;
-      g.i0 = i0; g.j0 = j0; g.causal = P.causal; g.window = P.window;
-      const bool any = (!P.causal || i0 <= j0 + 31) && (P.window == 0 || j0 - (i0 + 63) < P.window);
-      const bool full = (!P.causal || i0 + 63 <= j0) && (P.window == 0 || (j0 + 31) - i0 < P.window);
+      g.i0 = i0; g.j0 = j0; g.causal = P.causal; g.window = P.window; g.n = P.seqlen;
+      const bool any = j0 < P.seqlen && (!P.causal || i0 <= min(j0 + 31, P.seqlen - 1)) &&
+                       (P.window == 0 || j0 - (i0 + 63) < P.window);
+      const bool full = j0 + 31 < P.seqlen && i0 + 63 < P.seqlen && (!P.causal || i0 + 63 <= j0) &&
+                        (P.window == 0 || (j0 + 31) - i0 < P.window);
       float lam[4] = {1.0f, 1.0f, 1.0f, 1.0f};
       uint32_t flag = 0;
       unsigned long long cks[2] = {0ull, 0ull};
@@ -1264,9 +1269,9 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
       if (lane == 0) ptx::mbar_arrive(&bars[kPReady0 + grp]);
       LAMP_TOC(7, t_r);
 
-      const int64_t gt = (((int64_t)b * P.heads_q + h) * (P.seqlen / kBQ) + (j0 / kBQ)) * ntk + t;
-      if (lane == 0 && P.flag_mask) P.flag_mask[gt] = (uint8_t)flag;
-      if (DUMP && P.dbg_checksums) {
+      const int64_t gt = (((int64_t)b * P.heads_q + h) * ((P.seqlen + kBQ - 1) / kBQ) + (j0 / kBQ)) * ntk + t;
+      if (lane == 0 && P.flag_mask && j0 < P.seqlen) P.flag_mask[gt] = (uint8_t)flag;
+      if (DUMP && P.dbg_checksums && j0 < P.seqlen) {
 #pragma unroll
         for (int s = 16; s > 0; s >>= 1) {
           cks[0] += __shfl_xor_sync(kFull, cks[0], s);
@@ -1284,12 +1289,14 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
     for (int a = 1; a < 4; ++a)
       if ((lane & 3) == a) { om_row = st.om[a]; mu_row = st.mu[a]; }
     const int64_t orow = b * P.os[0] + h * P.os[1] + (int64_t)(j0 + lane) * P.os[2];
-    if (P.lse) P.lse[((int64_t)b * P.heads_q + h) * P.seqlen + j0 + lane] = (float)((double)mu_row + log((double)om_row));
+    const bool row_ok = j0 + lane < P.seqlen;   // rows past the end of the sequence are not stored
+    if (P.lse && row_ok) P.lse[((int64_t)b * P.heads_q + h) * P.seqlen + j0 + lane] = (float)((double)mu_row + log((double)om_row));
 #pragma unroll 1
     for (int c0 = 0; c0 < D; c0 += 16) {
       uint32_t r[16];
       ptx::tmem_ld16(tlane + c0, r);
       ptx::tmem_wait_ld();
+      if (!row_ok) continue;
       if (P.flags & LAMP_OUT_FP32) {
         float* dst = reinterpret_cast<float*>(P.out) + orow + c0;
 #pragma unroll

@@ -31,13 +31,14 @@ def compare_units(gpu, ref, *, check_stats=False, label=""):
         if ref.checks is not None and "checks" in gpu:
             gc = gpu["checks"][b, h, g].view(np.uint64)
             assert np.array_equal(gc, ref.checks[n]), f"{label} y8/e8 checksums differ at unit {(b, h, g)}"
+        nr = min(32, N - 32 * g)                 # the last group of a ragged sequence is partial
         go = gpu["out"][b, h, rows].astype(np.float64)
-        ro = ref.out[n].astype(np.float64)
+        ro = ref.out[n][:nr].astype(np.float64)
         assert np.isfinite(go).all()
         worst["o_abs"] = max(worst["o_abs"], float(np.abs(go - ro).max()))
         num += float(((go - ro) ** 2).sum()); den += float((ro ** 2).sum())
         gl = gpu["lse"][b, h, rows].astype(np.float64)
-        rl = ref.lse[n].astype(np.float64)
+        rl = ref.lse[n][:nr].astype(np.float64)
         worst["lse_abs"] = max(worst["lse_abs"], float(np.abs(gl - rl).max()))
         lnum += float(((gl - rl) ** 2).sum()); lden += float((rl ** 2).sum())
     worst["o_rel_fro"] = (num / max(den, 1e-300)) ** 0.5
@@ -57,5 +58,6 @@ def compare_dense_bytes(gpu, ref, b, h):
         if (ub, uh) != (b, h):
             continue
         rows = slice(32 * g, 32 * g + 32)
-        assert np.array_equal(gpu["y8"][rows], ref.y8[n]), f"y8 bytes differ in group {g}"
-        assert np.array_equal(gpu["e8"][rows], ref.e8[n]), f"e8 bytes differ in group {g}"
+        nr = min(32, gpu["y8"].shape[0] - 32 * g)
+        assert np.array_equal(gpu["y8"][rows], ref.y8[n][:nr]), f"y8 bytes differ in group {g}"
+        assert np.array_equal(gpu["e8"][rows], ref.e8[n][:nr]), f"e8 bytes differ in group {g}"

@@ -79,6 +79,24 @@ def test_masks(causal, window):
     compare_dense_bytes(gpu, ref, 0, 1)
 
 
+@pytest.mark.parametrize("N,causal,window,D,flags", [(200, True, 0, 128, 0), (161, True, 0, 128, 0), (97, True, 0, 128, 0),
+                                                     (333, False, 0, 128, 0), (300, True, 100, 128, 0),
+                                                     (1, True, 0, 128, 0), (65, True, 0, 256, 0),
+                                                     (250, True, 0, 256, 0), (190, True, 0, 128, oracle.FORCE_16BIT),
+                                                     (190, True, 0, 128, oracle.H16_SEQ), (131, False, 0, 128, oracle.FORCE_8BIT)])
+def test_ragged_sequence_lengths(N, causal, window, D, flags):
+    """Lengths that are not a multiple of the 32-row group, the 64-key tile or the 128-row CTA: rows and keys
+    past the end take part in nothing (votes, maxima, sums), nothing past the tensors is read or written."""
+    cfg = li.CONFIGS[1 if D == 128 else 3]
+    q, k, v = li.make_qkv(cfg, B=2, Hq=2, Hkv=1, N=N, seed=50 + N)
+    sc = li.softmax_scale(cfg.D)
+    ref = oracle.run_all(q, k, v, scale=sc, causal=causal, window=window, flags=flags, dumps=True)
+    gpu = run_gpu(q, k, v, scale=sc, causal=causal, window=window, flags=flags, dump=(1, 1))
+    assert gpu["out"].shape[2] == N and gpu["flags"].shape[2:] == ((N + 31) // 32, (N + 63) // 64)
+    compare_units(gpu, ref, check_stats=True, label=f"ragged N={N} causal={causal} window={window} D={D} flags={flags}")
+    compare_dense_bytes(gpu, ref, 1, 1)
+
+
 @pytest.mark.parametrize("mult", [0.5, 4.0, 8.0])
 def test_scale_sweep_saturation(mult):
     """Logit multipliers of the long-context sweep: at 4 and 8 many logits saturate at 448."""
@@ -212,9 +230,10 @@ def test_bad_arguments_are_rejected():
         lamp.forward(q, q, q, flags=lamp.LAMP_FORCE_16BIT | lamp.LAMP_FORCE_8BIT)
     with pytest.raises(lamp.LampAttnError):
         lamp.forward(q, q, q, causal=False, window=64)
-    q96 = torch.zeros(1, 2, 96, 128, device=dev, dtype=torch.bfloat16)
     with pytest.raises(lamp.LampAttnError):
-        lamp.forward(q96, q96, q96)
+        lamp.forward(q, q, q, flags=lamp.LAMP_SR_E4M3 | lamp.LAMP_H16_SEQ)
+    with pytest.raises(lamp.LampAttnError):
+        lamp.forward(q, q, q, threshold=-1.0)
     q64 = torch.zeros(1, 2, 128, 64, device=dev, dtype=torch.bfloat16)
     with pytest.raises(lamp.LampAttnError):
         lamp.forward(q64, q64, q64)
