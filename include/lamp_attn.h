@@ -140,7 +140,8 @@ size_t lamp_attn_workspace_bytes(const lamp_attn_params* p);
  *   workspace device scratch of at least lamp_attn_workspace_bytes(p) bytes (may be NULL
  *            when that is 0)
  *   cuda_stream a cudaStream_t (NULL = the default stream)
- * Inputs must be finite.  Logits beyond +-448 saturate (counted, not an error).
+ * Inputs must be finite.  Logits beyond +-448 saturate (counted, not an error).  batch = 0 or seqlen = 0 is an
+ * empty problem: LAMP_OK, nothing is enqueued and no pointer is looked at.
  * Errors: LAMP_ERR_INVALID_ARG, LAMP_ERR_UNSUPPORTED_SHAPE, LAMP_ERR_UNSUPPORTED_DEVICE,
  * LAMP_ERR_CUDA; nothing is enqueued when an error is returned. */
 int lamp_attn_fwd(const void* q, const void* k, const void* v, void* out, float* lse,

@@ -190,6 +190,9 @@ int lamp_attn_fwd(const void* q, const void* k, const void* v, void* out, float*
                   uint8_t* flag_mask, const lamp_attn_params* p, void* workspace,
                   size_t workspace_bytes, void* cuda_stream) {
   (void)workspace; (void)workspace_bytes;
+  // an empty problem (no batch entries or no tokens) is valid and enqueues nothing
+  if (p && (p->batch == 0 || p->seqlen == 0) && p->batch >= 0 && p->seqlen >= 0 && p->heads_q > 0 && p->heads_kv > 0)
+    return LAMP_OK;
   int rc = check_params(q, k, v, out, p);
   if (rc) return rc;
   int dev;

@@ -222,6 +222,15 @@ def test_strided_inputs_and_bf16_output():
     assert torch.equal(c["out"], b["out"].to(torch.bfloat16))
 
 
+def test_empty_problems_are_accepted():
+    import paper_2609_39361_b200 as lamp
+    dev = torch.device("cuda:0")
+    for shape in [(0, 2, 128, 128), (1, 2, 0, 128)]:
+        q = torch.zeros(*shape, device=dev, dtype=torch.bfloat16)
+        res = lamp.forward(q, q, q)
+        assert res["out"].shape == shape and res["flags"].numel() == 0
+
+
 def test_bad_arguments_are_rejected():
     import paper_2609_39361_b200 as lamp
     dev = torch.device("cuda:0")
