@@ -40,6 +40,8 @@ import lamp_inputs as li  # noqa: E402
 
 SM_COUNT, LANES_PER_SM, SM_MAX_MHZ = 148, 128, 1965.0
 MIN_SLOTS_PER_STEP = 2.0   # one FMA plus at least one instruction for the 8-bit rounding
+# the accumulation loop alone, measured in isolation: 3.56 cycles per warp-step and scheduler
+CHAIN_LOOP_PEAK = 4.0 * SM_COUNT * 4 * 32 * SM_MAX_MHZ * 1e6 / 3.56 / 1e12
 
 
 def valid_pairs(cfg, window=0):
@@ -324,7 +326,10 @@ def main():
     roofline = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                 "frac": achieved / peak, "traffic": traffic,
                 "note": "peak = issue-slot bound of the emulated e4m3 accumulation at 2 slots/step, "
-                        "148 SMs x 128 lanes x 1965 MHz (derived, not a measured peak)"}
+                        "148 SMs x 128 lanes x 1965 MHz (derived, not a measured peak); chain_loop_peak = the "
+                        "accumulation loop alone as measured on this GPU, 3.56 cycles per warp-step (packed FMA, "
+                        "two conversions and two f16->f32 share one pipe)",
+                "chain_loop_peak": CHAIN_LOOP_PEAK, "frac_of_chain_loop": achieved / CHAIN_LOOP_PEAK}
 
     cpu = None
     if not args.no_cpu_baseline:
