@@ -20,8 +20,8 @@
  * (each is listed, with the alternative, in the design notes of the repository):
  *   - rounding is round-to-nearest-even onto the real 8/16-bit grids, including
  *     their subnormals; overflow saturates to +-448 (Sec. 3.3 only prevents it);
- *   - the softmax scale is folded into Q once, in fp32 (Sec. 3.3 "applied before
- *     the matrix product is accumulated");
+ *   - the softmax scale is folded into Q once, in fp32 (Sec. 3.3 wants the 1/sqrt(d) scaling in
+ *     place before the accumulation starts);
  *   - a warp owns b_q = 32 query rows (Sec. 4.1 gives only b_q N_q = 128);
  *   - 16-bit logits are a sequential fp64 fma chain, rounded once to e4m11 (optional mode: the
  *     per-step e4m11 recursion instead);
@@ -36,7 +36,7 @@
 #include <stdlib.h>
 #include <string.h>
 
-#define BQ 32          /* query rows per warp (group)            Alg. 1 "single warp" */
+#define BQ 32          /* query rows per warp (group)            Alg. 1: the work of one warp */
 #define BK 16          /* keys per sub-block                     Sec. 4.1: 64 / N_k   */
 #define NK 4           /* sub-blocks per key tile                Sec. 4.1             */
 #define TK (BK * NK)   /* keys per tile                                                 */
@@ -94,7 +94,7 @@ float lamp_oracle_rne_e4m3(float x) { return (float)rne_grid((double)x, -6, 3, 4
 float lamp_oracle_rne_e4m11(double x) { return (float)rne_grid(x, -6, 11, 448.0); }
 
 /* Drop the low 8 mantissa bits of an e4m11 value (toward zero): Sec. 3.3,
- * "rounded to e4m3 ... by truncating the lower mantissa bits". */
+ * the running maxima reach the 8-bit shift by truncation of their low mantissa bits. */
 float lamp_oracle_trunc_e4m3(float x) {
   if (x == 0.0f || isinf(x)) return x;
   double a = fabs((double)x);
@@ -191,7 +191,7 @@ void lamp_oracle_exp16_array(const float* in, float* out, size_t n) {
 /* xi[theta][j]: per sub-block, per query sum of (omega_hat - e) e  (0 for sub-blocks
  * that are not free).  Returns the recompute set as a bitmask over theta: the
  * smallest set (then the smallest bitmask) whose removal makes every query's kept
- * sum <= tau * omega_hat^2.  Algorithm 1 "obtain solution g of block-LAMP problem". */
+ * sum <= tau * omega_hat^2.  The stage-2 step of Algorithm 1 (solve the block-LAMP problem). */
 uint32_t lamp_oracle_stage2(const double xi[NK][BQ], const float* omega_hat, float tau,
                             uint32_t free_mask) {
   for (int size = 0; size <= NK; ++size) {
@@ -215,9 +215,9 @@ float lamp_oracle_chain16(const float* a, const float* b, int n);
 float lamp_oracle_sr_e4m3(float t, uint32_t u20);
 uint32_t lamp_oracle_sr_bits(uint32_t seed, uint32_t bh, uint32_t j, uint32_t i, uint32_t kk);
 
-/* A 16-bit logit (Alg. 1 "recompute Y_theta in high precision").
+/* A 16-bit logit (the high-precision recomputation of a sub-block in Alg. 1).
  * Default reading: the exact dot product as a sequential fp64 fma chain over the channels, times the
- * scale, rounded once to e4m11 (Sec. 3.3 "a 16-bit e4m11 format to accumulate matrix products" taken as
+ * scale, rounded once to e4m11 (Sec. 3.3 names e4m11 as the 16-bit accumulation format; taken as
  * the format of the result).
  * LAMP_H16_SEQ, the other reading: the same recursion as the 8-bit pass (Sec. 4.1, round(c + a*b) with
  * the multiplication and addition in fp32), every partial sum rounded to e4m11, on the pre-scaled query. */
@@ -314,7 +314,7 @@ static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
       }
     if (!any) continue;
 
-    /* Alg. 1 "accumulate Y in low precision"; Sec. 4.1: round(c + a*b), fp32 fma. */
+    /* Alg. 1, low-precision accumulation of Y; Sec. 4.1: round(c + a*b), fp32 fma. */
     for (int i = 0; i < TK; ++i)
       for (int j = 0; j < BQ; ++j) {
         float c = 0.0f;

@@ -11,7 +11,7 @@
 
 namespace lamp {
 
-constexpr int kBQ = 32;   // query rows per warp ("single warp" of Alg. 1)
+constexpr int kBQ = 32;   // query rows per warp (the work of one warp in Alg. 1)
 constexpr int kBK = 16;   // keys per sub-block (Sec. 4.1: 64 keys / N_k = 4)
 constexpr int kNK = 4;    // sub-blocks per key tile
 constexpr int kTK = 64;   // keys per tile
@@ -49,7 +49,7 @@ __device__ __forceinline__ uint32_t enc_e4m3(float v) {
 }
 
 // Keep the top 3 mantissa bits of an e4m11 value, toward zero (Sec. 3.3: the running
-// maxima are "rounded to e4m3 ... by truncating the lower mantissa bits").
+// maxima reach the 8-bit shift by truncation of their low mantissa bits).
 __device__ __forceinline__ float trunc_e4m3(float x) {
   float a = fabsf(x);
   if (a < 0.015625f) return copysignf(truncf(a * 512.0f) * 0.001953125f, x);

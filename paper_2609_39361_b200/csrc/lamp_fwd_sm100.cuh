@@ -80,7 +80,7 @@ __device__ __forceinline__ void fma_x2(float& d0, float& d1, float a0, float a1,
 }
 
 // First pass: Y8[i][j] = chain over kk of c <- RNE_e4m3(fma(k, q*scale, c)), c0 = +0
-// (Alg. 1 "accumulate Y in low precision"; Sec. 4.1 round(c + a*b)), 128 channels per call.
+// (Alg. 1, low-precision accumulation of Y; Sec. 4.1 round(c + a*b)), 128 channels per call.
 // Operands of the next kk are fetched while the current one is processed; FMAs are issued
 // in packed pairs.  QF32: q holds fp32 q*scale, [kk][128 rows]; else raw bf16 q, scaled here
 // (one fp32 multiply, the same rounding).  FIRST: start from +0, else carry acc on.
@@ -380,7 +380,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 __device__ __forceinline__ uint32_t sw128(int row, int chunk) { return row * 128 + ((chunk ^ (row & 7)) << 4); }
 
 // Four e4m3 values <-> one 32-bit word (byte u = value u): the packed accumulator layout of
-// Sec. 3.3 ("4 accumulators occupy a single 32-bit register"), used to hand the first-pass
+// Sec. 3.3 (four 8-bit accumulators to a 32-bit register), used to hand the first-pass
 // logits from the chain warps to the decision-path warp through TMEM.  Exact both ways.
 __device__ __forceinline__ uint32_t pack_e4m3x4(float v0, float v1, float v2, float v3) {
   uint32_t r;
