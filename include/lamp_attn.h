@@ -39,7 +39,8 @@ typedef enum lamp_attn_error {
 } lamp_attn_error;
 
 /* Mode bits of lamp_attn_params.flags. */
-#define LAMP_FORCE_16BIT     0x01u /* every active sub-block takes the 16-bit path (comparison mode)      */
+#define LAMP_FORCE_16BIT     0x01u /* every active sub-block takes the 16-bit path (comparison mode); without
+                                      debug outputs the 8-bit pass is skipped and sat_e4m3 stays 0          */
 #define LAMP_FORCE_8BIT      0x02u /* no recomputation at all: the paper's pure 8-bit baseline (Sec. 4.1) */
 #define LAMP_NO_STAGE1       0x04u /* skip the running-maximum test (the paper's Appendix D ablation)     */
 #define LAMP_OUT_FP32        0x08u /* `out` is fp32 instead of bf16                                       */

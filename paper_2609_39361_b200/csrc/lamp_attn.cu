@@ -94,14 +94,15 @@ static int ensure_device(int* dev_out) {
     if (!fn || qr != cudaDriverEntryPointSuccess) return cuda_fail(cudaErrorNotSupported);
     g_encode = (TensorMapEncodeFn)fn;
   }
-  const void* kernels[12] = {
+  const void* kernels[14] = {
       (const void*)lamp_fwd_sm100<128, false, 0>, (const void*)lamp_fwd_sm100<128, true, 0>,
       (const void*)lamp_fwd_sm100<256, false, 0>, (const void*)lamp_fwd_sm100<256, true, 0>,
       (const void*)lamp_fwd_sm100<128, false, 1>, (const void*)lamp_fwd_sm100<128, true, 1>,
       (const void*)lamp_fwd_sm100<256, false, 1>, (const void*)lamp_fwd_sm100<256, true, 1>,
       (const void*)lamp_fwd_sm100<128, false, 2>, (const void*)lamp_fwd_sm100<128, true, 2>,
-      (const void*)lamp_fwd_sm100<256, false, 2>, (const void*)lamp_fwd_sm100<256, true, 2>};
-  for (int i = 0; i < 12; ++i) {
+      (const void*)lamp_fwd_sm100<256, false, 2>, (const void*)lamp_fwd_sm100<256, true, 2>,
+      (const void*)lamp_fwd_sm100<128, false, 3>, (const void*)lamp_fwd_sm100<256, false, 3>};
+  for (int i = 0; i < 14; ++i) {
     e = cudaFuncSetAttribute(kernels[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLaunch);
     if (e != cudaSuccess) return cuda_fail(e);
   }
@@ -247,10 +248,14 @@ int lamp_attn_fwd(const void* q, const void* k, const void* v, void* out, float*
   do {                                              \
     if (var == 0) LAMP_LAUNCH(D_, DUMP_, 0);        \
     else if (var == 1) LAMP_LAUNCH(D_, DUMP_, 1);   \
-    else LAMP_LAUNCH(D_, DUMP_, 2);                 \
+    else if (var == 2) LAMP_LAUNCH(D_, DUMP_, 2);   \
+    else LAMP_LAUNCH(D_, false, 3);                 \
   } while (0)
   // the per-step 16-bit accumulation (1) and the stochastic rounding (2) have kernels of their own
-  const int var = (p->flags & LAMP_H16_SEQ) ? 1 : (p->flags & LAMP_SR_E4M3) ? 2 : 0;
+  // ... and so has the all-16-bit comparison mode when nothing asks for the first-pass bytes (3: that pass is skipped,
+  // the counter of saturated first-pass maxima stays 0)
+  const int var = (p->flags & LAMP_H16_SEQ) ? 1 : (p->flags & LAMP_SR_E4M3) ? 2
+                  : ((p->flags & LAMP_FORCE_16BIT) && !dump) ? 3 : 0;
   if (p->head_dim == 128) {
     if (dump) LAMP_LAUNCH_VAR(128, true); else LAMP_LAUNCH_VAR(128, false);
   } else {

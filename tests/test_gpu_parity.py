@@ -161,6 +161,19 @@ def test_head_dim_256_gemma_shaped(window, flags):
     compare_dense_bytes(gpu, ref, 0, 1)
 
 
+@pytest.mark.parametrize("D,N,window", [(128, 640, 0), (256, 384, 0), (128, 300, 96)])
+def test_all_16bit_mode_without_the_first_pass(D, N, window):
+    """LAMP_FORCE_16BIT with no debug output skips the 8-bit pass altogether: outputs and flags must not change."""
+    cfg = li.CONFIGS[1 if D == 128 else 3]
+    q, k, v = li.make_qkv(cfg, B=1, Hq=4, Hkv=2, N=N, seed=77)
+    sc = li.softmax_scale(cfg.D)
+    ref = oracle.run_all(q, k, v, scale=sc, window=window, flags=oracle.FORCE_16BIT, checksums=False)
+    gpu = run_gpu(q, k, v, scale=sc, window=window, flags=oracle.FORCE_16BIT, checksums=False)
+    compare_units(gpu, ref, label=f"force16 fast D={D} N={N}")
+    st = gpu["stats"]
+    assert st["stage1_flagged"] == st["subblocks_active"] == ref.stats["subblocks_active"] and st["sat_e4m3"] == 0
+
+
 def test_config1_full():
     cfg = li.CONFIGS[1]
     q, k, v = li.make_qkv(cfg)
