@@ -106,13 +106,18 @@ __device__ __forceinline__ float rne_e4m11_f(float t) {
 
 // 16-bit exponential: exp(a) correctly rounded to 12 significant bits, with the
 // subnormal quantum 2^-41 below 2^-30 (ue5m11 with the bias that maps 0xF800 to 1.0).
-__device__ __forceinline__ float exp16(float a) {
+__device__ __forceinline__ float exp16(float a, double& as_double) {
   double v = exp((double)a);
   int e = ((__double2hiint(v) >> 20) & 0x7ff) - 1023;
   e = max(e, -30);
-  if (e > 900) return __int_as_float(0x7f800000);
+  if (e > 127) { as_double = __longlong_as_double(0x7ff0000000000000ll); return __int_as_float(0x7f800000); }   // beyond fp32
   double m = __hiloint2double(((e + 41 + 1023) << 20) | 0x00080000, 0);
-  return (float)__dsub_rn(__dadd_rn(v, m), m);
+  as_double = __dsub_rn(__dadd_rn(v, m), m);   // the rounded value, also wanted as a double for the row sums
+  return (float)as_double;
+}
+__device__ __forceinline__ float exp16(float a) {
+  double d;
+  return exp16(a, d);
 }
 
 // Index into the 256-entry table of Sec. 3.3: the non-negative shift rounded to 4

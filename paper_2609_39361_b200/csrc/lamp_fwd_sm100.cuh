@@ -611,11 +611,12 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
 #pragma unroll
       for (int b = 0; b < 4; ++b) {
         e[b] = 0.0f;
+        double ed = 0.0;
         if (vis<FULL>(g, 16 * th + 4 * th_own + b, 4 * qa + a)) {
-          e[b] = exp16(rne_sig12(__fsub_rn(__uint_as_float(y4[b]), mh)));
+          e[b] = exp16(rne_sig12(__fsub_rn(__uint_as_float(y4[b]), mh)), ed);
           wc.gt1 += e[b] > 1.0f;
         }
-        s += (double)e[b];
+        s += ed;
         h[b] = __bfloat162float(__float2bfloat16_rn(e[b]));
         l[b] = e[b] - h[b];
       }
