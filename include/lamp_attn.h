@@ -96,7 +96,9 @@ typedef struct lamp_attn_params {
   uint32_t reserved;                /* set to 0                                                  */
 } lamp_attn_params;
 
-/* Counters of the most recent lamp_attn_fwd on the current device. */
+/* Counters of the most recent lamp_attn_fwd on the current device.  They live in one block of device memory per
+ * GPU that every call clears when it starts: two calls whose kernels overlap (different streams, no ordering
+ * between them) mix their counts - the outputs are unaffected. */
 typedef struct lamp_attn_stats {
   uint64_t subblocks_active;         /* sub-blocks with at least one visible pair              */
   uint64_t stage1_flagged;           /* recomputed because eq. (7) failed                      */
