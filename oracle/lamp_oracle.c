@@ -55,6 +55,8 @@ typedef struct {
   float scale, tau, delta;
   uint32_t flags;
   uint32_t sr_seed;      /* seed of the counter-based generator of LAMP_SR_E4M3 */
+  int32_t group_rows;    /* b_q: query rows that decide together (a "warp" of Alg. 1); 0 = 32.  Sec. 4.1 fixes only
+                            b_q N_q = 128; 16 is the other instance offered, to bracket that reading */
 } lamp_oracle_params;
 
 typedef struct {
@@ -282,11 +284,12 @@ static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
                         uint8_t* e8d, lamp_oracle_stats* st) {
   const int D = p->head_dim, N = p->seqlen;
   const int hk = h / (p->heads_q / p->heads_kv);
-  const uint16_t* Q = q + ((int64_t)(b * p->heads_q + h) * N + (int64_t)g * BQ) * D;
+  const int bq = p->group_rows ? p->group_rows : BQ;   /* rows bq .. BQ-1 of the arrays below do not exist */
+  const uint16_t* Q = q + ((int64_t)(b * p->heads_q + h) * N + (int64_t)g * bq) * D;
   const uint16_t* K = k + (int64_t)(b * p->heads_kv + hk) * N * D;
   const uint16_t* V = v + (int64_t)(b * p->heads_kv + hk) * N * D;
   const int ntiles = (N + TK - 1) / TK;
-  const int64_t j0 = (int64_t)g * BQ;
+  const int64_t j0 = (int64_t)g * bq;
 
   float* qs = (float*)malloc(sizeof(float) * BQ * D);
   double* O = (double*)calloc((size_t)BQ * D, sizeof(double));
@@ -294,7 +297,7 @@ static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
   for (int j = 0; j < BQ; ++j) {
     mu[j] = -INFINITY;
     omega[j] = 0.0f;
-    for (int c = 0; c < D; ++c) qs[j * D + c] = j0 + j < N ? bf16_to_float(Q[j * D + c]) * p->scale : 0.0f;
+    for (int c = 0; c < D; ++c) qs[j * D + c] = (j < bq && j0 + j < N) ? bf16_to_float(Q[j * D + c]) * p->scale : 0.0f;
   }
   if (y8d) memset(y8d, 0x7F, (size_t)BQ * N);
   if (e8d) memset(e8d, 0xFF, (size_t)BQ * N);
@@ -309,7 +312,7 @@ static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
     int active[NK] = {0, 0, 0, 0}, any = 0;
     for (int i = 0; i < TK; ++i)
       for (int j = 0; j < BQ; ++j) {
-        val[i][j] = (uint8_t)pair_valid(p, i0 + i, j0 + j);
+        val[i][j] = (uint8_t)(j < bq && pair_valid(p, i0 + i, j0 + j));
         if (val[i][j]) active[i / BK] = 1, any = 1;
       }
     if (!any) continue;
@@ -496,7 +499,7 @@ static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
   }
 
   for (int j = 0; j < BQ; ++j) {
-    if (j0 + j >= N) {   /* rows past the end of a ragged sequence */
+    if (j >= bq || j0 + j >= N) {   /* rows that do not exist: past the group, or past a ragged sequence */
       for (int c = 0; c < D; ++c) out[j * D + c] = 0.0f;
       lse[j] = 0.0f;
       continue;
@@ -528,6 +531,7 @@ int lamp_oracle_units(const uint16_t* q, const uint16_t* k, const uint16_t* v,
                       float* out, float* lse, uint8_t* flags, uint64_t* checks, uint8_t* y8,
                       uint8_t* e8, lamp_oracle_stats* stats) {
   if (p->seqlen <= 0 || p->heads_q % p->heads_kv || p->head_dim <= 0 || p->head_dim > 256 ||
+      (p->group_rows != 0 && p->group_rows != 16 && p->group_rows != 32) ||
       p->delta < 0.0f || (p->window > 0 && !p->causal))
     return -1;
   const int N = p->seqlen, D = p->head_dim, nt = (N + TK - 1) / TK;

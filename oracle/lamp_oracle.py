@@ -27,7 +27,8 @@ class Params(C.Structure):
     _fields_ = [("batch", C.c_int32), ("heads_q", C.c_int32), ("heads_kv", C.c_int32),
                 ("seqlen", C.c_int32), ("head_dim", C.c_int32), ("causal", C.c_int32),
                 ("window", C.c_int32), ("scale", C.c_float), ("tau", C.c_float),
-                ("delta", C.c_float), ("flags", C.c_uint32), ("sr_seed", C.c_uint32)]
+                ("delta", C.c_float), ("flags", C.c_uint32), ("sr_seed", C.c_uint32),
+                ("group_rows", C.c_int32)]
 
 
 class Stats(C.Structure):
@@ -128,7 +129,7 @@ def _bits(x) -> np.ndarray:
 
 
 def run_units(q, k, v, units, *, causal=True, window=0, scale=None, tau=0.5, delta=2.0 ** -8,
-              flags=0, sr_seed=0, dumps=False, checksums=True) -> OracleResult:
+              flags=0, sr_seed=0, group_rows=0, dumps=False, checksums=True) -> OracleResult:
     """Run the oracle on the listed (b, h, g) units.  q: [B, Hq, N, D], k/v: [B, Hkv, N, D]."""
     qb, kb, vb = _bits(q), _bits(k), _bits(v)
     B, Hq, N, D = qb.shape
@@ -137,7 +138,7 @@ def run_units(q, k, v, units, *, causal=True, window=0, scale=None, tau=0.5, del
         scale = np.float32(1.0 / np.sqrt(float(D)))
     units = np.ascontiguousarray(np.asarray(units, dtype=np.int32).reshape(-1, 3))
     n = units.shape[0]
-    p = Params(B, Hq, Hkv, N, D, int(causal), int(window), float(scale), float(tau), float(delta), int(flags), int(sr_seed))
+    p = Params(B, Hq, Hkv, N, D, int(causal), int(window), float(scale), float(tau), float(delta), int(flags), int(sr_seed), int(group_rows))
     out = np.zeros((n, 32, D), np.float32)
     lse = np.zeros((n, 32), np.float32)
     fl = np.zeros((n, (N + 63) // 64), np.uint8)
@@ -153,12 +154,13 @@ def run_units(q, k, v, units, *, causal=True, window=0, scale=None, tau=0.5, del
     return OracleResult(units, out, lse, fl, ck, y8, e8, st.as_dict())
 
 
-def all_units(B, Hq, N):
-    g = np.stack(np.meshgrid(np.arange(B), np.arange(Hq), np.arange((N + 31) // 32), indexing="ij"), -1)
+def all_units(B, Hq, N, group_rows=32):
+    g = np.stack(np.meshgrid(np.arange(B), np.arange(Hq), np.arange((N + group_rows - 1) // group_rows),
+                             indexing="ij"), -1)
     return g.reshape(-1, 3).astype(np.int32)
 
 
 def run_all(q, k, v, **kw) -> OracleResult:
     qb = _bits(q)
     B, Hq, N, _ = qb.shape
-    return run_units(qb, k, v, all_units(B, Hq, N), **kw)
+    return run_units(qb, k, v, all_units(B, Hq, N, kw.get("group_rows", 0) or 32), **kw)

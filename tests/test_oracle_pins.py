@@ -429,6 +429,35 @@ def test_ragged_sequence_lengths():
             assert (got - o).abs().max() < 0.1 and (got - o).norm() / o.norm() < 5e-3
 
 
+def test_group_of_sixteen_rows(small):
+    """b_q = 16, the other instance of the group size Sec. 4.1 leaves open (b_q N_q = 128).  Pins: modes without
+    votes do not depend on the group size; with non-causal attention and every 16-row block repeated twice, a
+    32-row group votes exactly like its 16-row half; finer groups never recompute more."""
+    q, k, v, sc = small
+    for fl in (oracle.FORCE_8BIT, oracle.FORCE_16BIT):
+        a = oracle.run_all(q, k, v, scale=sc, flags=fl)
+        b = oracle.run_all(q, k, v, scale=sc, flags=fl, group_rows=16)
+        oa = a.out.reshape(1, 4, 16, 32, 128).reshape(1, 4, 512, 128)
+        ob = b.out.reshape(1, 4, 32, 32, 128)[:, :, :, :16].reshape(1, 4, 512, 128)
+        assert np.array_equal(oa, ob)
+        assert np.all(b.out.reshape(1, 4, 32, 32, 128)[:, :, :, 16:] == 0)
+    q2 = q.clone()
+    qv = q2.view(1, 4, 16, 2, 16, 128)
+    qv[:, :, :, 1] = qv[:, :, :, 0]                       # rows 16..31 of every 32-row block repeat rows 0..15
+    r32 = oracle.run_all(q2, k, v, scale=sc, causal=False)
+    r16 = oracle.run_all(q2, k, v, scale=sc, causal=False, group_rows=16)
+    f32 = r32.flags.reshape(4, 16, -1)
+    f16 = r16.flags.reshape(4, 32, -1)
+    assert np.array_equal(f16[:, 0::2], f32) and np.array_equal(f16[:, 1::2], f32)
+    o32 = r32.out.reshape(4, 16, 32, 128)
+    o16 = r16.out.reshape(4, 32, 32, 128)
+    assert np.array_equal(o16[:, 0::2, :16], o32[:, :, :16]) and np.array_equal(o16[:, 1::2, :16], o32[:, :, 16:])
+    p32 = oracle.run_all(q, k, v, scale=sc)
+    p16 = oracle.run_all(q, k, v, scale=sc, group_rows=16)
+    fr = lambda r: (r.stats["stage1_flagged"] + r.stats["stage2_flagged"]) / r.stats["subblocks_active"]
+    assert fr(p16) <= fr(p32)
+
+
 def test_rows_sum_to_one_and_units_are_independent(small):
     q, k, v, sc = small
     ones = torch.ones_like(v)
