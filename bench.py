@@ -7,7 +7,7 @@ input (B=4, 32 query / 8 KV heads, N=8192, head_dim 128, causal).  Prints ONE JS
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config C]
                   [--mode lamp|force8|force16] [--tau T] [--delta D] [--no-stage1]
-                  [--compact] [--h16-seq] [--sr] [--scale-mult M] [--window W]
+                  [--compact] [--h16-seq] [--sr] [--group-rows 16] [--scale-mult M] [--window W]
 
 The options after --config select the other workloads and the paper's ablations (threshold
 and margin sweeps, stage 1 off, the scale sweep of the long-context config, the sliding
@@ -134,7 +134,7 @@ def oracle_sample_run(cfg, q, k, v, scale, n_units, seed=11, knobs=None):
     t0 = time.perf_counter()
     oracle.run_units(q, k, v, units, scale=scale, causal=cfg.causal, window=window, tau=kn.get("tau", 0.5),
                      delta=kn.get("delta", 2.0 ** -8), flags=kn.get("flags", 0), sr_seed=kn.get("sr_seed", 0),
-                     checksums=False)
+                     group_rows=kn.get("group_rows", 0), checksums=False)
     dt = time.perf_counter() - t0
     fl = sum(4.0 * cfg.D * unit_pairs(cfg, int(g), window) for _, _, g in units)
     return dt, fl, len(units)
@@ -143,7 +143,8 @@ def oracle_sample_run(cfg, q, k, v, scale, n_units, seed=11, knobs=None):
 def knobs_of(args):
     """Thresholds, mode bits and mask of this run (the same numeric flag values in the library and the oracle)."""
     flags = {"lamp": 0, "force8": 2, "force16": 1}[args.mode] | (4 if args.no_stage1 else 0) | (16 if args.compact else 0) | (32 if args.h16_seq else 0) | (64 if args.sr else 0)
-    return {"tau": args.tau, "delta": args.delta, "flags": flags, "window": args.window, "sr_seed": args.sr_seed}
+    return {"tau": args.tau, "delta": args.delta, "flags": flags, "window": args.window, "sr_seed": args.sr_seed,
+            "group_rows": args.group_rows}
 
 
 def reference_arm(args, cfg, rank):
@@ -191,6 +192,8 @@ def workload_config(cfg, args):
         extra += ", per-step e4m11 accumulation"
     if args.sr:
         extra += f", stochastic rounding (seed {args.sr_seed})"
+    if args.group_rows != 32:
+        extra += f", groups of {args.group_rows} rows"
     return {"workload": f"config {cfg.index}: {cfg.name} prefill, B={cfg.B}, Hq={cfg.Hq}, Hkv={cfg.Hkv}, "
                         f"N={cfg.N}, head_dim={cfg.D}, causal{extra}, tau={args.tau:g}, delta=2^{math.log2(args.delta):g}",
             "l2": "inputs (Q+K+V+O = %.0f MB) larger than the 126 MB L2" %
@@ -217,6 +220,8 @@ def main():
     ap.add_argument("--sr", action="store_true",
                     help="stochastic rounding in the 8-bit accumulation (Sec. 3.3), counter-based generator")
     ap.add_argument("--sr-seed", type=int, default=1)
+    ap.add_argument("--group-rows", type=int, default=32, choices=[16, 32],
+                    help="b_q: query rows that decide together (the paper fixes only b_q N_q = 128)")
     ap.add_argument("--scale-mult", type=float, default=1.0, help="softmax scale = mult / sqrt(head_dim)")
     ap.add_argument("--window", type=int, default=0, help="sliding window (0 = global causal)")
     args = ap.parse_args()
@@ -247,18 +252,20 @@ def main():
 
     scale = li.softmax_scale(cfg.D, args.scale_mult)
     kn = knobs_of(args)
+    GR = args.group_rows
     q, k, v = li.make_qkv(cfg)
     hq, hk, hv = q.pin_memory(), k.pin_memory(), v.pin_memory()
     dq, dk, dv = hq.to(dev), hk.to(dev), hv.to(dev)
     B, Hq, N, D = q.shape
     out = torch.empty(B, Hq, N, D, device=dev, dtype=torch.bfloat16)
     lse = torch.empty(B, Hq, N, device=dev, dtype=torch.float32)
-    fm = torch.empty(B, Hq, N // 32, N // 64, device=dev, dtype=torch.uint8)
+    fm = torch.empty(B, Hq, N // GR, N // 64, device=dev, dtype=torch.uint8)
     p = lamp.lamp_attn_default_params()
     p.batch, p.heads_q, p.heads_kv, p.seqlen, p.head_dim = B, Hq, k.shape[1], N, D
     lamp.lamp_attn_contiguous_strides(p)
     p.causal, p.window, p.scale = 1, args.window, scale
     p.threshold, p.delta, p.flags, p.sr_seed = args.tau, args.delta, kn["flags"], args.sr_seed
+    p.group_rows = args.group_rows
     fl = flops_of(cfg, args.window)
 
     def step():
@@ -286,7 +293,7 @@ def main():
     # ---- end to end: pinned host inputs in, result out, every step -------------------------
     ho = torch.empty(B, Hq, N, D, dtype=torch.bfloat16).pin_memory()
     hl = torch.empty(B, Hq, N, dtype=torch.float32).pin_memory()
-    hf = torch.empty(B, Hq, N // 32, N // 64, dtype=torch.uint8).pin_memory()
+    hf = torch.empty(B, Hq, N // GR, N // 64, dtype=torch.uint8).pin_memory()
 
     def e2e_step():
         dq.copy_(hq, non_blocking=True); dk.copy_(hk, non_blocking=True); dv.copy_(hv, non_blocking=True)
@@ -320,7 +327,7 @@ def main():
     peak = 4.0 / MIN_SLOTS_PER_STEP * SM_COUNT * LANES_PER_SM * SM_MAX_MHZ * 1e6 / 1e12
     # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu capture summarised in
     # profiles/lamp_fwd_sm100_config2_ncu_full.txt (algorithmic bytes: 680 MB)
-    headline = (args.mode == "lamp" and not args.no_stage1 and not args.compact and not args.h16_seq and not args.sr and args.tau == 0.5 and args.delta == 2.0 ** -8
+    headline = (args.mode == "lamp" and not args.no_stage1 and not args.compact and not args.h16_seq and not args.sr and args.group_rows == 32 and args.tau == 0.5 and args.delta == 2.0 ** -8
                 and args.scale_mult == 1.0 and args.window == 0)
     traffic = {2: 657.16e6}.get(cfg.index) if headline else None
     roofline = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",

@@ -93,7 +93,11 @@ typedef struct lamp_attn_params {
   uint64_t* dbg_checksums;          /* [batch, heads_q, seqlen/32, seqlen/64, 2]: position-keyed
                                        checksums of the y8 and e8 bytes of each (group, tile)  */
   uint32_t sr_seed;                 /* seed of the generator of LAMP_SR_E4M3 (unused otherwise)  */
-  uint32_t reserved;                /* set to 0                                                  */
+  int32_t group_rows;               /* b_q, the query rows that decide together (one warp of Alg. 1): 0 or
+                                       32 (Sec. 4.1 fixes only b_q N_q = 128; this library's reading), or 16, the
+                                       other instance on offer: flag_mask and dbg_checksums then have seqlen/16
+                                       groups, the kernel runs at half its efficiency, and the modes
+                                       LAMP_SR_E4M3 and LAMP_H16_SEQ are not available                     */
 } lamp_attn_params;
 
 /* Counters of the most recent lamp_attn_fwd on the current device.  They live in one block of device memory per

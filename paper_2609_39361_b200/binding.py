@@ -26,7 +26,7 @@ class LampAttnParams(C.Structure):
                 ("threshold", C.c_float), ("delta", C.c_float), ("flags", C.c_uint32),
                 ("dbg_batch", C.c_int32), ("dbg_head", C.c_int32),
                 ("dbg_y8", C.c_void_p), ("dbg_e8", C.c_void_p), ("dbg_checksums", C.c_void_p),
-                ("sr_seed", C.c_uint32), ("reserved", C.c_uint32)]
+                ("sr_seed", C.c_uint32), ("group_rows", C.c_int32)]
 
 
 class LampAttnStats(C.Structure):
@@ -164,7 +164,7 @@ def lamp_attn_get_stats(stream=None) -> dict:
 
 
 def forward(q, k, v, *, causal=True, window=0, scale=None, threshold=0.5, delta=2.0 ** -8, flags=0, sr_seed=0,
-            out_fp32=False, want_lse=True, want_flags=True, dump=None, checksums=False, stream=None):
+            group_rows=0, out_fp32=False, want_lse=True, want_flags=True, dump=None, checksums=False, stream=None):
     """Convenience wrapper: allocate outputs with torch, fill the params struct, call
     ``lamp_attn_fwd``.  q: [B, Hq, N, D] bf16 CUDA; k, v: [B, Hkv, N, D].
     dump=(batch, head) also returns the dense y8 / e8 byte maps of that head."""
@@ -183,16 +183,18 @@ def forward(q, k, v, *, causal=True, window=0, scale=None, threshold=0.5, delta=
     p.threshold, p.delta = float(threshold), float(delta)
     p.flags = int(flags) | (LAMP_OUT_FP32 if out_fp32 else 0)
     p.sr_seed = int(sr_seed)
+    p.group_rows = int(group_rows)
+    gr = int(group_rows) or 32
     res = {"out": out}
     lse = torch.empty(B, Hq, N, device=q.device, dtype=torch.float32) if want_lse else None
-    fm = torch.empty(B, Hq, (N + 31) // 32, (N + 63) // 64, device=q.device, dtype=torch.uint8) if want_flags else None
+    fm = torch.empty(B, Hq, (N + gr - 1) // gr, (N + 63) // 64, device=q.device, dtype=torch.uint8) if want_flags else None
     if dump is not None:
         p.dbg_batch, p.dbg_head = dump
         res["y8"] = torch.full((N, N), 0x7F, device=q.device, dtype=torch.uint8)
         res["e8"] = torch.full((N, N), 0xFF, device=q.device, dtype=torch.uint8)
         p.dbg_y8, p.dbg_e8 = res["y8"].data_ptr(), res["e8"].data_ptr()
     if checksums:
-        res["checks"] = torch.empty(B, Hq, (N + 31) // 32, (N + 63) // 64, 2, device=q.device, dtype=torch.int64)
+        res["checks"] = torch.empty(B, Hq, (N + gr - 1) // gr, (N + 63) // 64, 2, device=q.device, dtype=torch.int64)
         p.dbg_checksums = res["checks"].data_ptr()
     ws_bytes = lamp_attn_workspace_bytes(p)
     ws = torch.empty(ws_bytes, device=q.device, dtype=torch.uint8) if ws_bytes else None

@@ -94,15 +94,17 @@ static int ensure_device(int* dev_out) {
     if (!fn || qr != cudaDriverEntryPointSuccess) return cuda_fail(cudaErrorNotSupported);
     g_encode = (TensorMapEncodeFn)fn;
   }
-  const void* kernels[14] = {
+  const void* kernels[18] = {
       (const void*)lamp_fwd_sm100<128, false, 0>, (const void*)lamp_fwd_sm100<128, true, 0>,
       (const void*)lamp_fwd_sm100<256, false, 0>, (const void*)lamp_fwd_sm100<256, true, 0>,
       (const void*)lamp_fwd_sm100<128, false, 1>, (const void*)lamp_fwd_sm100<128, true, 1>,
       (const void*)lamp_fwd_sm100<256, false, 1>, (const void*)lamp_fwd_sm100<256, true, 1>,
       (const void*)lamp_fwd_sm100<128, false, 2>, (const void*)lamp_fwd_sm100<128, true, 2>,
       (const void*)lamp_fwd_sm100<256, false, 2>, (const void*)lamp_fwd_sm100<256, true, 2>,
-      (const void*)lamp_fwd_sm100<128, false, 3>, (const void*)lamp_fwd_sm100<256, false, 3>};
-  for (int i = 0; i < 14; ++i) {
+      (const void*)lamp_fwd_sm100<128, false, 3>, (const void*)lamp_fwd_sm100<256, false, 3>,
+      (const void*)lamp_fwd_sm100<128, false, 4>, (const void*)lamp_fwd_sm100<128, true, 4>,
+      (const void*)lamp_fwd_sm100<256, false, 4>, (const void*)lamp_fwd_sm100<256, true, 4>};
+  for (int i = 0; i < 18; ++i) {
     e = cudaFuncSetAttribute(kernels[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLaunch);
     if (e != cudaSuccess) return cuda_fail(e);
   }
@@ -174,6 +176,8 @@ static int check_params(const void* q, const void* k, const void* v, void* out,
   if ((p->flags & LAMP_FORCE_16BIT) && (p->flags & (LAMP_FORCE_8BIT | LAMP_NO_STAGE1)))
     return LAMP_ERR_INVALID_ARG;
   if ((p->flags & LAMP_SR_E4M3) && (p->flags & LAMP_H16_SEQ)) return LAMP_ERR_INVALID_ARG;
+  if (p->group_rows != 0 && p->group_rows != 16 && p->group_rows != 32) return LAMP_ERR_INVALID_ARG;
+  if (p->group_rows == 16 && (p->flags & (LAMP_SR_E4M3 | LAMP_H16_SEQ))) return LAMP_ERR_INVALID_ARG;
   if ((p->dbg_y8 || p->dbg_e8) &&
       (p->dbg_batch < 0 || p->dbg_batch >= p->batch || p->dbg_head < 0 || p->dbg_head >= p->heads_q))
     return LAMP_ERR_INVALID_ARG;
@@ -211,6 +215,7 @@ int lamp_attn_fwd(const void* q, const void* k, const void* v, void* out, float*
   P.batch = p->batch; P.heads_q = p->heads_q; P.heads_kv = p->heads_kv; P.seqlen = p->seqlen;
   P.causal = p->causal ? 1 : 0; P.window = p->window;
   P.scale = p->scale; P.tau = p->threshold; P.delta = p->delta; P.flags = p->flags; P.sr_seed = p->sr_seed;
+  P.group_rows = p->group_rows ? p->group_rows : kBQ;
   P.dbg_batch = p->dbg_batch; P.dbg_head = p->dbg_head;
   P.dbg_y8 = p->dbg_y8; P.dbg_e8 = p->dbg_e8;
   P.dbg_checksums = (unsigned long long*)p->dbg_checksums;
@@ -221,7 +226,8 @@ int lamp_attn_fwd(const void* q, const void* k, const void* v, void* out, float*
   e = cudaMemsetAsync(stats_ptr, 0, sizeof(DeviceStats), stream);
   if (e != cudaSuccess) return cuda_fail(e);
 
-  const size_t ngt = (size_t)p->batch * p->heads_q * ((p->seqlen + kBQ - 1) / kBQ) * ((p->seqlen + kTK - 1) / kTK);
+  const int bq = p->group_rows ? p->group_rows : kBQ;
+  const size_t ngt = (size_t)p->batch * p->heads_q * ((p->seqlen + bq - 1) / bq) * ((p->seqlen + kTK - 1) / kTK);
   if (flag_mask) {
     e = cudaMemsetAsync(flag_mask, 0, ngt, stream);
     if (e != cudaSuccess) return cuda_fail(e);
@@ -239,7 +245,7 @@ int lamp_attn_fwd(const void* q, const void* k, const void* v, void* out, float*
   rc = make_kv_map(&vmap, v, p->v_strides, p->head_dim, p->seqlen, p->heads_kv, p->batch);
   if (rc) return rc;
   const bool dump = p->dbg_y8 || p->dbg_e8 || p->dbg_checksums;
-  dim3 grid((p->seqlen + kBM - 1) / kBM, p->heads_q, p->batch), block(kThreads);
+  dim3 grid((p->seqlen + 4 * bq - 1) / (4 * bq), p->heads_q, p->batch), block(kThreads);
   const uint2* lutp = (const uint2*)lut_ptr;
   DeviceStats* dsp = (DeviceStats*)stats_ptr;
 #define LAMP_LAUNCH(D_, DUMP_, VAR_) \
@@ -249,12 +255,13 @@ int lamp_attn_fwd(const void* q, const void* k, const void* v, void* out, float*
     if (var == 0) LAMP_LAUNCH(D_, DUMP_, 0);        \
     else if (var == 1) LAMP_LAUNCH(D_, DUMP_, 1);   \
     else if (var == 2) LAMP_LAUNCH(D_, DUMP_, 2);   \
+    else if (var == 4) LAMP_LAUNCH(D_, DUMP_, 4);   \
     else LAMP_LAUNCH(D_, false, 3);                 \
   } while (0)
   // the per-step 16-bit accumulation (1) and the stochastic rounding (2) have kernels of their own
   // ... and so has the all-16-bit comparison mode when nothing asks for the first-pass bytes (3: that pass is skipped,
   // the counter of saturated first-pass maxima stays 0)
-  const int var = (p->flags & LAMP_H16_SEQ) ? 1 : (p->flags & LAMP_SR_E4M3) ? 2
+  const int var = bq == 16 ? 4 : (p->flags & LAMP_H16_SEQ) ? 1 : (p->flags & LAMP_SR_E4M3) ? 2
                   : ((p->flags & LAMP_FORCE_16BIT) && !dump) ? 3 : 0;
   if (p->head_dim == 128) {
     if (dump) LAMP_LAUNCH_VAR(128, true); else LAMP_LAUNCH_VAR(128, false);
@@ -322,7 +329,8 @@ int lamp_attn_fwd_digest(const void* q, const void* k, const void* v, void* out,
   if (!p || !digest) return LAMP_ERR_INVALID_ARG;
   if (p->batch <= 0 || p->heads_q <= 0 || p->seqlen <= 0) return LAMP_ERR_INVALID_ARG;
   const unsigned long long n_pairs =
-      (unsigned long long)p->batch * p->heads_q * ((p->seqlen + kBQ - 1) / kBQ) * ((p->seqlen + kTK - 1) / kTK);
+      (unsigned long long)p->batch * p->heads_q * ((p->seqlen + (p->group_rows ? p->group_rows : kBQ) - 1) / (p->group_rows ? p->group_rows : kBQ)) *
+      ((p->seqlen + kTK - 1) / kTK);
   if (n_pairs > LAMP_DIGEST_MAX_PAIRS) return LAMP_ERR_UNSUPPORTED_SHAPE;   // beyond the built-in scratch
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);

@@ -166,6 +166,7 @@ struct KernelParams {
   float scale, tau, delta;
   uint32_t flags;
   uint32_t sr_seed;
+  int group_rows;
   int dbg_batch, dbg_head;
   uint8_t* dbg_y8;
   uint8_t* dbg_e8;

@@ -67,10 +67,11 @@ enum Bar {
 
 struct TileGeom {
   int i0, j0, causal, window, n;   // n: sequence length (rows and keys past it do not exist)
+  int bq;                          // rows of the group that exist (32, or 16 for the smaller group size)
 };
 template <bool FULL>
 __device__ __forceinline__ bool vis(const TileGeom& g, int i, int j) {
-  return FULL || (g.i0 + i < g.n && g.j0 + j < g.n && pair_valid(g.causal, g.window, g.i0 + i, g.j0 + j));
+  return FULL || (j < g.bq && g.i0 + i < g.n && g.j0 + j < g.n && pair_valid(g.causal, g.window, g.i0 + i, g.j0 + j));
 }
 
 __device__ __forceinline__ void fma_x2(float& d0, float& d1, float a0, float a1, uint64_t bb, float c0, float c1) {
@@ -490,7 +491,7 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
     bool act = true;
     if (!FULL) {
       const int s0 = g.i0 + 16 * th;
-      act = s0 < g.n && (!g.causal || s0 <= min(g.j0 + 31, g.n - 1)) && (g.window == 0 || g.j0 - (s0 + 15) < g.window);
+      act = s0 < g.n && (!g.causal || s0 <= min(g.j0 + g.bq - 1, g.n - 1)) && (g.window == 0 || g.j0 - (s0 + 15) < g.window);
     }
     actmask |= (uint32_t)act << th;
   }
@@ -879,7 +880,8 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
 
 
 // VAR 1: the per-step reading of the 16-bit accumulation (mode LAMP_H16_SEQ); VAR 2: stochastic rounding in
-// the first pass (mode LAMP_SR_E4M3); VAR 3: LAMP_FORCE_16BIT without debug outputs, the first pass skipped.  Kernels of their own, so that the default one (VAR 0) carries nothing
+// the first pass (mode LAMP_SR_E4M3); VAR 3: LAMP_FORCE_16BIT without debug outputs, the first pass skipped;
+// VAR 4: groups of 16 instead of 32 rows (group_rows = 16).  Kernels of their own, so that the default one (VAR 0) carries nothing
 // of them (code that never ran still cost it 2.5 % through register allocation).
 template <int D, bool DUMP, int VAR>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -906,14 +908,16 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
   int* status = &gstats->status;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int ntq = (P.seqlen + kBM - 1) / kBM;
+  constexpr int bq = (VAR == 4) ? 16 : kBQ;    // 32, or 16: then rows 16..31 of every group of lanes do not exist
+  const int cta_rows = 4 * bq;                 // query rows of one CTA
+  const int ntq = (P.seqlen + cta_rows - 1) / cta_rows;
   const int qt = ntq - 1 - (int)blockIdx.x;   // long (late) query tiles first
   const int h = blockIdx.y, b = blockIdx.z;
   const int hk = h / (P.heads_q / P.heads_kv);
-  const int m0 = qt * kBM;
+  const int m0 = qt * cta_rows;
 
   int t_begin = 0, t_end = (P.seqlen + kTK - 1) / kTK;
-  if (P.causal) t_end = min(t_end, (min(m0 + kBM, P.seqlen) - 1) / kTK + 1);
+  if (P.causal) t_end = min(t_end, (min(m0 + cta_rows, P.seqlen) - 1) / kTK + 1);
   if (P.window > 0) t_begin = max(0, m0 - P.window + 1) / kTK;
   const int T = t_end - t_begin;
   const int M = T * NH;                       // half-tiles of the K (and V) stream
@@ -952,7 +956,8 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
     const __nv_bfloat16* qg = P.q + b * P.qs[0] + h * P.qs[1] + (int64_t)m0 * P.qs[2];
     for (int c = tid; c < kBM * D / 8; c += kThreads) {
       const int row = c % kBM, k0 = (c / kBM) * 8;   // consecutive threads -> consecutive rows
-      const int rsrc = min(row, P.seqlen - 1 - m0);  // rows past the end of the sequence repeat the last one (never used)
+      // rows past the group (smaller group size) or past the sequence repeat the last one (never used)
+      const int rsrc = min((row >> 5) * bq + min(row & 31, bq - 1), P.seqlen - 1 - m0);
       const uint4 raw = *reinterpret_cast<const uint4*>(qg + (int64_t)rsrc * P.qs[2] + k0);
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
@@ -1092,13 +1097,13 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
     asm volatile("setmaxnreg.dec.sync.aligned.u32 120;");
     const int grp = warp & 3, side = (warp >> 2) - 1;   // side 0: even tiles, side 1: odd tiles
     const int qa = lane >> 2;
-    const int j0 = m0 + grp * kBQ;
+    const int j0 = m0 + grp * bq;
     const uint32_t tring = tbase + ((uint32_t)(grp * 32) << 16) + kColRing;
     const unsigned char* q_quad = qs + (QF32 ? 4 : 2) * (grp * kBQ + 4 * qa);
     bool ok = true;
     for (int n = side; n < T && ok; n += 2) {
       const int i0 = (t_begin + n) * kTK;
-      const bool any = j0 < P.seqlen && (!P.causal || i0 <= min(j0 + 31, P.seqlen - 1)) &&
+      const bool any = j0 < P.seqlen && (!P.causal || i0 <= min(j0 + bq - 1, P.seqlen - 1)) &&
                        (P.window == 0 || j0 - (i0 + 63) < P.window);
       float acc[4][16];
 #pragma unroll
@@ -1150,7 +1155,7 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
     asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
     const int grp = warp;
     const int qa = lane >> 2;
-    const int j0 = m0 + grp * kBQ;
+    const int j0 = m0 + grp * bq;
     const int ntk = (P.seqlen + kTK - 1) / kTK;
     const bool dump_rows = DUMP && b == P.dbg_batch && h == P.dbg_head;
     const __nv_bfloat16* kg = P.k + b * P.ks[0] + hk * P.ks[1];
@@ -1159,7 +1164,7 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
     const uint32_t tlane = tbase + ((uint32_t)(grp * 32) << 16);
     const uint32_t tscr = tlane + kColScr, tq = tlane + kColQ, tring = tlane + kColRing;
     {
-      const __nv_bfloat16* qrow = P.q + b * P.qs[0] + h * P.qs[1] + (int64_t)min(j0 + lane, P.seqlen - 1) * P.qs[2];
+      const __nv_bfloat16* qrow = P.q + b * P.qs[0] + h * P.qs[1] + (int64_t)min(j0 + min(lane, bq - 1), P.seqlen - 1) * P.qs[2];
 #pragma unroll 1
       for (int c0 = 0; c0 < 128; c0 += 16) {
         uint32_t r[16];
@@ -1194,10 +1199,10 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
     for (int n = 0; n < T && ok; ++n) {
       const int t = t_begin + n, i0 = t * kTK;
       TileGeom g;
-      g.i0 = i0; g.j0 = j0; g.causal = P.causal; g.window = P.window; g.n = P.seqlen;
-      const bool any = j0 < P.seqlen && (!P.causal || i0 <= min(j0 + 31, P.seqlen - 1)) &&
+      g.i0 = i0; g.j0 = j0; g.causal = P.causal; g.window = P.window; g.n = P.seqlen; g.bq = bq;
+      const bool any = j0 < P.seqlen && (!P.causal || i0 <= min(j0 + bq - 1, P.seqlen - 1)) &&
                        (P.window == 0 || j0 - (i0 + 63) < P.window);
-      const bool full = j0 + 31 < P.seqlen && i0 + 63 < P.seqlen && (!P.causal || i0 + 63 <= j0) &&
+      const bool full = bq == kBQ && j0 + 31 < P.seqlen && i0 + 63 < P.seqlen && (!P.causal || i0 + 63 <= j0) &&
                         (P.window == 0 || (j0 + 31) - i0 < P.window);
       float lam[4] = {1.0f, 1.0f, 1.0f, 1.0f};
       uint32_t flag = 0;
@@ -1272,7 +1277,7 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
       if (lane == 0) ptx::mbar_arrive(&bars[kPReady0 + grp]);
       LAMP_TOC(7, t_r);
 
-      const int64_t gt = (((int64_t)b * P.heads_q + h) * ((P.seqlen + kBQ - 1) / kBQ) + (j0 / kBQ)) * ntk + t;
+      const int64_t gt = (((int64_t)b * P.heads_q + h) * ((P.seqlen + bq - 1) / bq) + (j0 / bq)) * ntk + t;
       if (lane == 0 && P.flag_mask && j0 < P.seqlen) P.flag_mask[gt] = (uint8_t)flag;
       if (DUMP && P.dbg_checksums && j0 < P.seqlen) {
 #pragma unroll
@@ -1292,7 +1297,7 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
     for (int a = 1; a < 4; ++a)
       if ((lane & 3) == a) { om_row = st.om[a]; mu_row = st.mu[a]; }
     const int64_t orow = b * P.os[0] + h * P.os[1] + (int64_t)(j0 + lane) * P.os[2];
-    const bool row_ok = j0 + lane < P.seqlen;   // rows past the end of the sequence are not stored
+    const bool row_ok = lane < bq && j0 + lane < P.seqlen;   // rows past the group or the sequence are not stored
     if (P.lse && row_ok) P.lse[((int64_t)b * P.heads_q + h) * P.seqlen + j0 + lane] = (float)((double)mu_row + log((double)om_row));
 #pragma unroll 1
     for (int c0 = 0; c0 < D; c0 += 16) {

@@ -19,19 +19,19 @@ def run_gpu(q, k, v, *, dump=None, checksums=True, **kw):
     return out
 
 
-def compare_units(gpu, ref, *, check_stats=False, label=""):
+def compare_units(gpu, ref, *, check_stats=False, label="", bq=32):
     """gpu: dict from run_gpu (dense arrays); ref: OracleResult for a list of units."""
     N = gpu["out"].shape[2]
     worst = {"o_abs": 0.0, "lse_abs": 0.0}
     num = den = lnum = lden = 0.0
     for n, (b, h, g) in enumerate(ref.units):
-        rows = slice(32 * g, 32 * g + 32)
+        rows = slice(bq * g, bq * g + bq)
         gf = gpu["flags"][b, h, g]
         assert np.array_equal(gf, ref.flags[n]), f"{label} flag bytes differ at unit {(b, h, g)}: {gf} vs {ref.flags[n]}"
         if ref.checks is not None and "checks" in gpu:
             gc = gpu["checks"][b, h, g].view(np.uint64)
             assert np.array_equal(gc, ref.checks[n]), f"{label} y8/e8 checksums differ at unit {(b, h, g)}"
-        nr = min(32, N - 32 * g)                 # the last group of a ragged sequence is partial
+        nr = min(bq, N - bq * g)                 # the last group of a ragged sequence is partial
         go = gpu["out"][b, h, rows].astype(np.float64)
         ro = ref.out[n][:nr].astype(np.float64)
         assert np.isfinite(go).all()
@@ -52,12 +52,12 @@ def compare_units(gpu, ref, *, check_stats=False, label=""):
     return worst
 
 
-def compare_dense_bytes(gpu, ref, b, h):
+def compare_dense_bytes(gpu, ref, b, h, bq=32):
     """Dense y8 / e8 maps of head (b, h) against the oracle's per-unit dumps."""
     for n, (ub, uh, g) in enumerate(ref.units):
         if (ub, uh) != (b, h):
             continue
-        rows = slice(32 * g, 32 * g + 32)
-        nr = min(32, gpu["y8"].shape[0] - 32 * g)
+        rows = slice(bq * g, bq * g + bq)
+        nr = min(bq, gpu["y8"].shape[0] - bq * g)
         assert np.array_equal(gpu["y8"][rows], ref.y8[n][:nr]), f"y8 bytes differ in group {g}"
         assert np.array_equal(gpu["e8"][rows], ref.e8[n][:nr]), f"e8 bytes differ in group {g}"
