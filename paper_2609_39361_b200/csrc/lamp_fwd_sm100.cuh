@@ -319,7 +319,6 @@ __device__ __noinline__ void dot16_seq(const __nv_bfloat16* __restrict__ krow, i
   for (int a = 0; a < 4; ++a)
 #pragma unroll
     for (int b = 0; b < 4; ++b) acc[a][b] = 0.0f;
-  const __nv_bfloat16* ksrc = krow + (int64_t)(4 * tp) * kstride;
   uint4 kraw[4];
 #pragma unroll
   for (int b = 0; b < 4; ++b) kraw[b] = *reinterpret_cast<const uint4*>(krow + (int64_t)min(4 * tp + b, nkey - 1) * kstride);
