@@ -37,6 +37,7 @@
 #include <string.h>
 
 #define BQ 32          /* query rows per warp (group)            Alg. 1: the work of one warp */
+#define BQM 64         /* the largest group size on offer (group_rows = 64); sizes of the per-unit arrays */
 #define BK 16          /* keys per sub-block                     Sec. 4.1: 64 / N_k   */
 #define NK 4           /* sub-blocks per key tile                Sec. 4.1             */
 #define TK (BK * NK)   /* keys per tile                                                 */
@@ -194,16 +195,16 @@ void lamp_oracle_exp16_array(const float* in, float* out, size_t n) {
  * that are not free).  Returns the recompute set as a bitmask over theta: the
  * smallest set (then the smallest bitmask) whose removal makes every query's kept
  * sum <= tau * omega_hat^2.  The stage-2 step of Algorithm 1 (solve the block-LAMP problem). */
-uint32_t lamp_oracle_stage2(const double xi[NK][BQ], const float* omega_hat, float tau,
+static uint32_t stage2_rows(const double* xi, int ld, int nrows, const float* omega_hat, float tau,
                             uint32_t free_mask) {
   for (int size = 0; size <= NK; ++size) {
     for (uint32_t r = 0; r < (1u << NK); ++r) {
       if ((r & ~free_mask) != 0 || __builtin_popcount(r) != size) continue;
       int ok = 1;
-      for (int j = 0; j < BQ && ok; ++j) {
+      for (int j = 0; j < nrows && ok; ++j) {
         double kept = 0.0;
         for (int th = 0; th < NK; ++th)
-          if (((free_mask & ~r) >> th) & 1u) kept += xi[th][j];
+          if (((free_mask & ~r) >> th) & 1u) kept += xi[th * ld + j];
         double rhs = ((double)tau * (double)omega_hat[j]) * (double)omega_hat[j];
         if (!(kept <= rhs)) ok = 0;
       }
@@ -211,6 +212,10 @@ uint32_t lamp_oracle_stage2(const double xi[NK][BQ], const float* omega_hat, flo
     }
   }
   return free_mask;
+}
+uint32_t lamp_oracle_stage2(const double xi[NK][BQ], const float* omega_hat, float tau,
+                            uint32_t free_mask) {
+  return stage2_rows(&xi[0][0], BQ, BQ, omega_hat, tau, free_mask);
 }
 
 float lamp_oracle_chain16(const float* a, const float* b, int n);
@@ -252,7 +257,7 @@ static uint64_t mix64(uint64_t x) {
  * from a recomputed logit far above the running maximum; then a plain double sum is
  * used and the event is reported.)  *big is set when the sum reaches 2^12, beyond
  * which a double no longer holds it exactly. */
-static double exact_rowsum(const float Ef[TK][BQ], int j, int* big) {
+static double exact_rowsum(const float Ef[TK][BQM], int j, int* big) {
   unsigned __int128 acc = 0;
   int huge = 0;
   double plain = 0.0;
@@ -284,26 +289,27 @@ static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
                         uint8_t* e8d, lamp_oracle_stats* st) {
   const int D = p->head_dim, N = p->seqlen;
   const int hk = h / (p->heads_q / p->heads_kv);
-  const int bq = p->group_rows ? p->group_rows : BQ;   /* rows bq .. BQ-1 of the arrays below do not exist */
+  const int bq = p->group_rows ? p->group_rows : BQ;   /* rows bq .. BQM-1 of the arrays below do not exist */
+  const int bqo = bq > BQ ? BQM : BQ;                  /* rows per unit in the output arrays */
   const uint16_t* Q = q + ((int64_t)(b * p->heads_q + h) * N + (int64_t)g * bq) * D;
   const uint16_t* K = k + (int64_t)(b * p->heads_kv + hk) * N * D;
   const uint16_t* V = v + (int64_t)(b * p->heads_kv + hk) * N * D;
   const int ntiles = (N + TK - 1) / TK;
   const int64_t j0 = (int64_t)g * bq;
 
-  float* qs = (float*)malloc(sizeof(float) * BQ * D);
-  double* O = (double*)calloc((size_t)BQ * D, sizeof(double));
-  float mu[BQ], omega[BQ];
-  for (int j = 0; j < BQ; ++j) {
+  float* qs = (float*)malloc(sizeof(float) * BQM * D);
+  double* O = (double*)calloc((size_t)BQM * D, sizeof(double));
+  float mu[BQM], omega[BQM];
+  for (int j = 0; j < BQM; ++j) {
     mu[j] = -INFINITY;
     omega[j] = 0.0f;
     for (int c = 0; c < D; ++c) qs[j * D + c] = (j < bq && j0 + j < N) ? bf16_to_float(Q[j * D + c]) * p->scale : 0.0f;
   }
-  if (y8d) memset(y8d, 0x7F, (size_t)BQ * N);
-  if (e8d) memset(e8d, 0xFF, (size_t)BQ * N);
+  if (y8d) memset(y8d, 0x7F, (size_t)bqo * N);
+  if (e8d) memset(e8d, 0xFF, (size_t)bqo * N);
 
-  float Y8[TK][BQ], Y16[TK][BQ], Ef[TK][BQ];
-  uint8_t E8[TK][BQ], val[TK][BQ];
+  float Y8[TK][BQM], Y16[TK][BQM], Ef[TK][BQM];
+  uint8_t E8[TK][BQM], val[TK][BQM];
 
   for (int t = 0; t < ntiles; ++t) {
     const int64_t i0 = (int64_t)t * TK;
@@ -311,7 +317,7 @@ static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
     if (checks) checks[2 * t] = checks[2 * t + 1] = 0;
     int active[NK] = {0, 0, 0, 0}, any = 0;
     for (int i = 0; i < TK; ++i)
-      for (int j = 0; j < BQ; ++j) {
+      for (int j = 0; j < BQM; ++j) {
         val[i][j] = (uint8_t)(j < bq && pair_valid(p, i0 + i, j0 + j));
         if (val[i][j]) active[i / BK] = 1, any = 1;
       }
@@ -319,7 +325,7 @@ static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
 
     /* Alg. 1, low-precision accumulation of Y; Sec. 4.1: round(c + a*b), fp32 fma. */
     for (int i = 0; i < TK; ++i)
-      for (int j = 0; j < BQ; ++j) {
+      for (int j = 0; j < BQM; ++j) {
         float c = 0.0f;
         if (!val[i][j]) { Y8[i][j] = 0.0f; continue; }   /* never used, and may lie past the tensors */
         for (int kk = 0; kk < D; ++kk)
@@ -335,9 +341,9 @@ static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
       }
 
     /* maximum low-precision logit per sub-block and query (the C matrix of Sec. 3.1) */
-    float cm8[NK][BQ];
+    float cm8[NK][BQM];
     for (int th = 0; th < NK; ++th)
-      for (int j = 0; j < BQ; ++j) {
+      for (int j = 0; j < BQM; ++j) {
         float m = -INFINITY;
         for (int i = th * BK; i < (th + 1) * BK; ++i)
           if (val[i][j] && Y8[i][j] > m) m = Y8[i][j];
@@ -350,7 +356,7 @@ static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
     int order[NK], nact = 0;
     for (int th = 0; th < NK; ++th) {
       T[th] = -INFINITY;
-      for (int j = 0; j < BQ; ++j)
+      for (int j = 0; j < BQM; ++j)
         if (cm8[th][j] > -INFINITY) {
           float d = cm8[th][j] - mu[j];
           if (d > T[th]) T[th] = d;
@@ -364,7 +370,7 @@ static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
     }
 
     /* stage 1: eq. (7) on the running maxima, sub-blocks in threat order */
-    float muh[BQ];
+    float muh[BQM];
     memcpy(muh, mu, sizeof(mu));
     uint32_t Theta = 0;
     const int skip1 = (p->flags & (LAMP_FORCE_8BIT | LAMP_NO_STAGE1)) != 0;
@@ -373,7 +379,7 @@ static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
       int pass = 1;
       if (p->flags & LAMP_FORCE_16BIT) pass = 0;
       else if (!skip1)
-        for (int j = 0; j < BQ; ++j) {
+        for (int j = 0; j < BQM; ++j) {
           if (!(cm8[th][j] > -INFINITY)) continue;
           if (isinf(muh[j])) { pass = 0; break; }
           float margin = fabsf(muh[j]) * p->delta;
@@ -383,7 +389,7 @@ static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
       if (pass) continue;
       Theta |= 1u << th;
       for (int i = th * BK; i < (th + 1) * BK; ++i)
-        for (int j = 0; j < BQ; ++j) {
+        for (int j = 0; j < BQM; ++j) {
           if (!val[i][j]) continue;
           Y16[i][j] = logit16(p, K + (size_t)(i0 + i) * D, Q + (size_t)j * D, qs + (size_t)j * D, D);
           if (fabsf(Y16[i][j]) == 448.0f) st->sat_e4m11++;
@@ -391,13 +397,13 @@ static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
         }
     }
     if (skip1)
-      for (int j = 0; j < BQ; ++j)
+      for (int j = 0; j < BQM; ++j)
         for (int th = 0; th < NK; ++th)
           if (cm8[th][j] > muh[j]) muh[j] = cm8[th][j];
 
     /* exponentials: 8-bit through the table, 16-bit correctly rounded */
     for (int i = 0; i < TK; ++i)
-      for (int j = 0; j < BQ; ++j) {
+      for (int j = 0; j < BQM; ++j) {
         Ef[i][j] = 0.0f;
         E8[i][j] = 0xFF;
         if (!val[i][j]) continue;
@@ -414,13 +420,13 @@ static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
       }
 
     /* lambda_hat (high precision), exact row sums, omega_hat */
-    float lam[BQ], omh[BQ];
-    for (int j = 0; j < BQ; ++j) {
+    float lam[BQM], omh[BQM];
+    for (int j = 0; j < BQM; ++j) {
       float d = mu[j] - muh[j];
       lam[j] = isinf(mu[j]) ? 0.0f : (float)exp((double)d);
     }
     int bigrow = 0;
-    for (int j = 0; j < BQ; ++j)
+    for (int j = 0; j < BQM; ++j)
       omh[j] = (float)((double)lam[j] * (double)omega[j] + exact_rowsum(Ef, j, &bigrow));
 
     /* stage 2: block-LAMP problem, eq. (8) */
@@ -428,16 +434,16 @@ static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
     for (int th = 0; th < NK; ++th)
       if (active[th] && !((Theta >> th) & 1u)) freem |= 1u << th;
     if (!(p->flags & (LAMP_FORCE_8BIT | LAMP_FORCE_16BIT)) && freem) {
-      double xi[NK][BQ];
+      double xi[NK][BQM];
       for (int th = 0; th < NK; ++th)
-        for (int j = 0; j < BQ; ++j) {
+        for (int j = 0; j < BQM; ++j) {
           double s = 0.0;
           if ((freem >> th) & 1u)
             for (int i = th * BK; i < (th + 1) * BK; ++i)
               if (val[i][j]) s += ((double)omh[j] - (double)Ef[i][j]) * (double)Ef[i][j];
           xi[th][j] = s;
         }
-      Rset = lamp_oracle_stage2(xi, omh, p->tau, freem);
+      Rset = stage2_rows(&xi[0][0], BQM, BQM, omh, p->tau, freem);
     }
     /* Compact register layout (Sec. 3.3, "Register layout"): when the two stages mark two or more
      * sub-blocks of the tile, the update of O falls back to 16 bits for the whole tile.  Reading taken
@@ -447,13 +453,13 @@ static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
 
     /* dumps and checksums refer to the 8-bit pass before any stage-2 replacement */
     for (int i = 0; i < TK; ++i)
-      for (int j = 0; j < BQ; ++j) {
+      for (int j = 0; j < BQM; ++j) {
         if (!val[i][j]) continue;
         uint8_t yb = lamp_oracle_enc_e4m3(Y8[i][j]);
         if (y8d) y8d[(size_t)j * N + i0 + i] = yb;
         if (e8d) e8d[(size_t)j * N + i0 + i] = E8[i][j];
         if (checks) {
-          uint64_t idx = (uint64_t)(i * BQ + j) << 8;
+          uint64_t idx = (uint64_t)(i * bqo + j) << 8;
           checks[2 * t] += mix64(idx | yb);
           checks[2 * t + 1] += mix64(idx | E8[i][j]);
         }
@@ -463,7 +469,7 @@ static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
     for (int th = 0; th < NK; ++th) {
       if (!((Rset >> th) & 1u)) continue;
       for (int i = th * BK; i < (th + 1) * BK; ++i)
-        for (int j = 0; j < BQ; ++j) {
+        for (int j = 0; j < BQM; ++j) {
           if (!val[i][j]) continue;
           float y = logit16(p, K + (size_t)(i0 + i) * D, Q + (size_t)j * D, qs + (size_t)j * D, D);
           if (fabsf(y) == 448.0f) st->sat_e4m11++;
@@ -474,11 +480,11 @@ static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
     }
 
     /* state update and P V (fp64 here) */
-    float omn[BQ];
-    for (int j = 0; j < BQ; ++j)
+    float omn[BQM];
+    for (int j = 0; j < BQM; ++j)
       omn[j] = (float)((double)lam[j] * (double)omega[j] + exact_rowsum(Ef, j, &bigrow));
     if (bigrow) st->big_rowsum++;
-    for (int j = 0; j < BQ; ++j) {
+    for (int j = 0; j < BQM; ++j) {
       mu[j] = muh[j];
       omega[j] = omn[j];
       for (int c = 0; c < D; ++c) O[j * D + c] *= (double)lam[j];
@@ -498,7 +504,7 @@ static void oracle_unit(const uint16_t* q, const uint16_t* k, const uint16_t* v,
     st->hist_flagged_per_tile[__builtin_popcount(Theta | Rset)]++;
   }
 
-  for (int j = 0; j < BQ; ++j) {
+  for (int j = 0; j < bqo; ++j) {
     if (j >= bq || j0 + j >= N) {   /* rows that do not exist: past the group, or past a ragged sequence */
       for (int c = 0; c < D; ++c) out[j * D + c] = 0.0f;
       lse[j] = 0.0f;
@@ -531,10 +537,11 @@ int lamp_oracle_units(const uint16_t* q, const uint16_t* k, const uint16_t* v,
                       float* out, float* lse, uint8_t* flags, uint64_t* checks, uint8_t* y8,
                       uint8_t* e8, lamp_oracle_stats* stats) {
   if (p->seqlen <= 0 || p->heads_q % p->heads_kv || p->head_dim <= 0 || p->head_dim > 256 ||
-      (p->group_rows != 0 && p->group_rows != 16 && p->group_rows != 32) ||
+      (p->group_rows != 0 && p->group_rows != 16 && p->group_rows != 32 && p->group_rows != 64) ||
       p->delta < 0.0f || (p->window > 0 && !p->causal))
     return -1;
   const int N = p->seqlen, D = p->head_dim, nt = (N + TK - 1) / TK;
+  const int bqo = p->group_rows > BQ ? BQM : BQ;   /* rows per unit in out, lse, y8, e8 */
   lamp_oracle_stats total;
   memset(&total, 0, sizeof(total));
   for (int i = 0; i < 256; ++i) g_lut8[i] = lamp_oracle_lut8((uint8_t)i);
@@ -545,9 +552,9 @@ int lamp_oracle_units(const uint16_t* q, const uint16_t* k, const uint16_t* v,
 #pragma omp for schedule(dynamic, 1)
     for (int64_t u = 0; u < n_units; ++u)
       oracle_unit(q, k, v, p, units[3 * u], units[3 * u + 1], units[3 * u + 2],
-                  out + (size_t)u * BQ * D, lse + (size_t)u * BQ, flags + (size_t)u * nt,
-                  checks ? checks + (size_t)u * nt * 2 : NULL, y8 ? y8 + (size_t)u * BQ * N : NULL,
-                  e8 ? e8 + (size_t)u * BQ * N : NULL, &mine);
+                  out + (size_t)u * bqo * D, lse + (size_t)u * bqo, flags + (size_t)u * nt,
+                  checks ? checks + (size_t)u * nt * 2 : NULL, y8 ? y8 + (size_t)u * bqo * N : NULL,
+                  e8 ? e8 + (size_t)u * bqo * N : NULL, &mine);
 #pragma omp critical
     stats_add(&total, &mine);
   }

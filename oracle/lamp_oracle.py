@@ -139,12 +139,13 @@ def run_units(q, k, v, units, *, causal=True, window=0, scale=None, tau=0.5, del
     units = np.ascontiguousarray(np.asarray(units, dtype=np.int32).reshape(-1, 3))
     n = units.shape[0]
     p = Params(B, Hq, Hkv, N, D, int(causal), int(window), float(scale), float(tau), float(delta), int(flags), int(sr_seed), int(group_rows))
-    out = np.zeros((n, 32, D), np.float32)
-    lse = np.zeros((n, 32), np.float32)
+    rows = 64 if int(group_rows) > 32 else 32          # rows per unit in the outputs
+    out = np.zeros((n, rows, D), np.float32)
+    lse = np.zeros((n, rows), np.float32)
     fl = np.zeros((n, (N + 63) // 64), np.uint8)
     ck = np.zeros((n, (N + 63) // 64, 2), np.uint64) if checksums else None
-    y8 = np.zeros((n, 32, N), np.uint8) if dumps else None
-    e8 = np.zeros((n, 32, N), np.uint8) if dumps else None
+    y8 = np.zeros((n, rows, N), np.uint8) if dumps else None
+    e8 = np.zeros((n, rows, N), np.uint8) if dumps else None
     st = Stats()
     ptr = lambda a: a.ctypes.data_as(C.c_void_p) if a is not None else None
     rc = lib().lamp_oracle_units(ptr(qb), ptr(kb), ptr(vb), C.byref(p), n, ptr(units), ptr(out),

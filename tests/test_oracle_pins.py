@@ -458,6 +458,32 @@ def test_group_of_sixteen_rows(small):
     assert fr(p16) <= fr(p32)
 
 
+def test_group_of_sixty_four_rows(small):
+    """b_q = 64 (two warps of rows deciding together), the same pins: vote-free modes agree row by row with
+    b_q = 32; with non-causal attention and every 32-row block repeated twice a 64-row group decides like its
+    32-row half; coarser groups never recompute less."""
+    q, k, v, sc = small
+    for fl in (oracle.FORCE_8BIT, oracle.FORCE_16BIT):
+        a = oracle.run_all(q, k, v, scale=sc, flags=fl)
+        b = oracle.run_all(q, k, v, scale=sc, flags=fl, group_rows=64)
+        assert b.out.shape == (4 * 8, 64, 128)
+        assert np.array_equal(a.out.reshape(1, 4, 512, 128), b.out.reshape(1, 4, 512, 128))
+        assert np.array_equal(a.lse.reshape(1, 4, 512), b.lse.reshape(1, 4, 512))
+    q2 = q.clone()
+    qv = q2.view(1, 4, 8, 2, 32, 128)
+    qv[:, :, :, 1] = qv[:, :, :, 0]
+    r32 = oracle.run_all(q2, k, v, scale=sc, causal=False)
+    r64 = oracle.run_all(q2, k, v, scale=sc, causal=False, group_rows=64)
+    f32 = r32.flags.reshape(4, 16, -1)
+    f64 = r64.flags.reshape(4, 8, -1)
+    assert np.array_equal(f32[:, 0::2], f64) and np.array_equal(f32[:, 1::2], f64)
+    assert np.array_equal(r32.out.reshape(4, 512, 128), r64.out.reshape(4, 512, 128))
+    p32 = oracle.run_all(q, k, v, scale=sc)
+    p64 = oracle.run_all(q, k, v, scale=sc, group_rows=64)
+    fr = lambda r: (r.stats["stage1_flagged"] + r.stats["stage2_flagged"]) / r.stats["subblocks_active"]
+    assert fr(p64) >= fr(p32)
+
+
 def test_rows_sum_to_one_and_units_are_independent(small):
     q, k, v, sc = small
     ones = torch.ones_like(v)
