@@ -220,7 +220,7 @@ def main():
     ap.add_argument("--sr", action="store_true",
                     help="stochastic rounding in the 8-bit accumulation (Sec. 3.3), counter-based generator")
     ap.add_argument("--sr-seed", type=int, default=1)
-    ap.add_argument("--group-rows", type=int, default=32, choices=[16, 32],
+    ap.add_argument("--group-rows", type=int, default=32, choices=[16, 32, 64],
                     help="b_q: query rows that decide together (the paper fixes only b_q N_q = 128)")
     ap.add_argument("--scale-mult", type=float, default=1.0, help="softmax scale = mult / sqrt(head_dim)")
     ap.add_argument("--window", type=int, default=0, help="sliding window (0 = global causal)")

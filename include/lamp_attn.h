@@ -94,10 +94,11 @@ typedef struct lamp_attn_params {
                                        checksums of the y8 and e8 bytes of each (group, tile)  */
   uint32_t sr_seed;                 /* seed of the generator of LAMP_SR_E4M3 (unused otherwise)  */
   int32_t group_rows;               /* b_q, the query rows that decide together (one warp of Alg. 1): 0 or
-                                       32 (Sec. 4.1 fixes only b_q N_q = 128; this library's reading), or 16, the
-                                       other instance on offer: flag_mask and dbg_checksums then have seqlen/16
-                                       groups, the kernel runs at half its efficiency, and the modes
-                                       LAMP_SR_E4M3 and LAMP_H16_SEQ are not available                     */
+                                       32 (Sec. 4.1 fixes only b_q N_q = 128; this library's reading), or the
+                                       other two instances: 16 (the kernel runs at half its efficiency) and 64
+                                       (two warps exchange their votes through shared memory).  flag_mask and
+                                       dbg_checksums then have seqlen/16 resp. seqlen/64 groups; the modes
+                                       LAMP_SR_E4M3 and LAMP_H16_SEQ are not available with 16 or 64        */
 } lamp_attn_params;
 
 /* Counters of the most recent lamp_attn_fwd on the current device.  They live in one block of device memory per

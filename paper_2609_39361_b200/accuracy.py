@@ -55,6 +55,7 @@ MODES = [
     ("lamp compact branch", lamp.LAMP_COMPACT_BRANCH, {}),
     ("lamp per-step e4m11", lamp.LAMP_H16_SEQ, {}),
     ("lamp groups of 16 rows", 0, {"group_rows": 16}),
+    ("lamp groups of 64 rows", 0, {"group_rows": 64}),
     ("force16", lamp.LAMP_FORCE_16BIT, {}),
     ("force8 stochastic", lamp.LAMP_FORCE_8BIT | lamp.LAMP_SR_E4M3, {"sr_seed": 1}),
     ("lamp stochastic", lamp.LAMP_SR_E4M3, {"sr_seed": 1}),

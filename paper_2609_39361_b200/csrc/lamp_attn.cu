@@ -94,7 +94,7 @@ static int ensure_device(int* dev_out) {
     if (!fn || qr != cudaDriverEntryPointSuccess) return cuda_fail(cudaErrorNotSupported);
     g_encode = (TensorMapEncodeFn)fn;
   }
-  const void* kernels[18] = {
+  const void* kernels[22] = {
       (const void*)lamp_fwd_sm100<128, false, 0>, (const void*)lamp_fwd_sm100<128, true, 0>,
       (const void*)lamp_fwd_sm100<256, false, 0>, (const void*)lamp_fwd_sm100<256, true, 0>,
       (const void*)lamp_fwd_sm100<128, false, 1>, (const void*)lamp_fwd_sm100<128, true, 1>,
@@ -103,8 +103,10 @@ static int ensure_device(int* dev_out) {
       (const void*)lamp_fwd_sm100<256, false, 2>, (const void*)lamp_fwd_sm100<256, true, 2>,
       (const void*)lamp_fwd_sm100<128, false, 3>, (const void*)lamp_fwd_sm100<256, false, 3>,
       (const void*)lamp_fwd_sm100<128, false, 4>, (const void*)lamp_fwd_sm100<128, true, 4>,
-      (const void*)lamp_fwd_sm100<256, false, 4>, (const void*)lamp_fwd_sm100<256, true, 4>};
-  for (int i = 0; i < 18; ++i) {
+      (const void*)lamp_fwd_sm100<256, false, 4>, (const void*)lamp_fwd_sm100<256, true, 4>,
+      (const void*)lamp_fwd_sm100<128, false, 5>, (const void*)lamp_fwd_sm100<128, true, 5>,
+      (const void*)lamp_fwd_sm100<256, false, 5>, (const void*)lamp_fwd_sm100<256, true, 5>};
+  for (int i = 0; i < 22; ++i) {
     e = cudaFuncSetAttribute(kernels[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLaunch);
     if (e != cudaSuccess) return cuda_fail(e);
   }
@@ -176,8 +178,8 @@ static int check_params(const void* q, const void* k, const void* v, void* out,
   if ((p->flags & LAMP_FORCE_16BIT) && (p->flags & (LAMP_FORCE_8BIT | LAMP_NO_STAGE1)))
     return LAMP_ERR_INVALID_ARG;
   if ((p->flags & LAMP_SR_E4M3) && (p->flags & LAMP_H16_SEQ)) return LAMP_ERR_INVALID_ARG;
-  if (p->group_rows != 0 && p->group_rows != 16 && p->group_rows != 32) return LAMP_ERR_INVALID_ARG;
-  if (p->group_rows == 16 && (p->flags & (LAMP_SR_E4M3 | LAMP_H16_SEQ))) return LAMP_ERR_INVALID_ARG;
+  if (p->group_rows != 0 && p->group_rows != 16 && p->group_rows != 32 && p->group_rows != 64) return LAMP_ERR_INVALID_ARG;
+  if ((p->group_rows == 16 || p->group_rows == 64) && (p->flags & (LAMP_SR_E4M3 | LAMP_H16_SEQ))) return LAMP_ERR_INVALID_ARG;
   if ((p->dbg_y8 || p->dbg_e8) &&
       (p->dbg_batch < 0 || p->dbg_batch >= p->batch || p->dbg_head < 0 || p->dbg_head >= p->heads_q))
     return LAMP_ERR_INVALID_ARG;
@@ -245,7 +247,8 @@ int lamp_attn_fwd(const void* q, const void* k, const void* v, void* out, float*
   rc = make_kv_map(&vmap, v, p->v_strides, p->head_dim, p->seqlen, p->heads_kv, p->batch);
   if (rc) return rc;
   const bool dump = p->dbg_y8 || p->dbg_e8 || p->dbg_checksums;
-  dim3 grid((p->seqlen + 4 * bq - 1) / (4 * bq), p->heads_q, p->batch), block(kThreads);
+  const int cta_rows = bq == 16 ? 64 : 128;
+  dim3 grid((p->seqlen + cta_rows - 1) / cta_rows, p->heads_q, p->batch), block(kThreads);
   const uint2* lutp = (const uint2*)lut_ptr;
   DeviceStats* dsp = (DeviceStats*)stats_ptr;
 #define LAMP_LAUNCH(D_, DUMP_, VAR_) \
@@ -256,12 +259,13 @@ int lamp_attn_fwd(const void* q, const void* k, const void* v, void* out, float*
     else if (var == 1) LAMP_LAUNCH(D_, DUMP_, 1);   \
     else if (var == 2) LAMP_LAUNCH(D_, DUMP_, 2);   \
     else if (var == 4) LAMP_LAUNCH(D_, DUMP_, 4);   \
+    else if (var == 5) LAMP_LAUNCH(D_, DUMP_, 5);   \
     else LAMP_LAUNCH(D_, false, 3);                 \
   } while (0)
   // the per-step 16-bit accumulation (1) and the stochastic rounding (2) have kernels of their own
   // ... and so has the all-16-bit comparison mode when nothing asks for the first-pass bytes (3: that pass is skipped,
   // the counter of saturated first-pass maxima stays 0)
-  const int var = bq == 16 ? 4 : (p->flags & LAMP_H16_SEQ) ? 1 : (p->flags & LAMP_SR_E4M3) ? 2
+  const int var = bq == 16 ? 4 : bq == 64 ? 5 : (p->flags & LAMP_H16_SEQ) ? 1 : (p->flags & LAMP_SR_E4M3) ? 2
                   : ((p->flags & LAMP_FORCE_16BIT) && !dump) ? 3 : 0;
   if (p->head_dim == 128) {
     if (dump) LAMP_LAUNCH_VAR(128, true); else LAMP_LAUNCH_VAR(128, false);

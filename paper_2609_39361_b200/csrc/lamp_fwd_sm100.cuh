@@ -47,7 +47,8 @@ struct SmemLayout {
   static constexpr int kDscr = kLut + 2048;                       // 4 groups x 384 doubles
   static constexpr int kBar = kDscr + 4 * 384 * 8;                // mbarriers
   static constexpr int kMisc = kBar + 512;                        // tmem slot, lo masks
-  static constexpr int kBytes = kMisc + 64;
+  static constexpr int kPairX = kMisc + 64;                       // 2 pairs x 2 slots x 2 warps x 16 bytes
+  static constexpr int kBytes = kPairX + 128;
   static_assert(kKbf % 1024 == 0 && kV % 1024 == 0 && kPhi % 1024 == 0 && kPlo % 1024 == 0, "swizzle atoms");
 };
 
@@ -62,16 +63,43 @@ enum Bar {
   kSlotPad = kPvDone0 + 4,
   kSlotFull0 = kSlotPad,                   // [group][slot]: a packed chain tile waits in TMEM
   kSlotEmpty0 = kSlotFull0 + 4 * kSlots,   // [group][slot]: the decision-path warp has taken it
-  kNumBars = kSlotEmpty0 + 4 * kSlots
+  kPairBar0 = kSlotEmpty0 + 4 * kSlots,    // [pair]: both decision-path warps of a 64-row group have published
+  kNumBars = kPairBar0 + 2
 };
+static_assert(kNumBars * 8 <= 512, "barrier area");
 
 struct TileGeom {
   int i0, j0, causal, window, n;   // n: sequence length (rows and keys past it do not exist)
-  int bq;                          // rows of the group that exist (32, or 16 for the smaller group size)
+  int bq;                          // rows of the warp that exist (32, or 16 for the smaller group size)
+  int gj0, gbq;                    // first row and size of the deciding group (= j0, bq unless two warps decide together)
 };
 template <bool FULL>
 __device__ __forceinline__ bool vis(const TileGeom& g, int i, int j) {
   return FULL || (j < g.bq && g.i0 + i < g.n && g.j0 + j < g.n && pair_valid(g.causal, g.window, g.i0 + i, g.j0 + j));
+}
+
+// Groups of 64 rows (group_rows = 64): the two decision-path warps of a pair vote together.  A warp publishes a
+// warp-uniform 16-byte value in shared memory, arrives on the pair's mbarrier and reads the partner's value once
+// both have arrived (two slots alternate, so a fast warp cannot overwrite what the partner still reads; the
+// wait is bounded like every other).  Both warps run the same number of exchanges per tile by construction:
+// every branch that contains one depends only on values the pair shares.
+struct PairX {
+  uint4* slots;      // [2 slots][2 warps]
+  uint64_t* bar;     // count 2
+  uint32_t seq;
+  int w;             // which warp of the pair
+  int* status;
+};
+__device__ __forceinline__ uint4 pair_exchange(PairX& px, uint4 mine, bool& ok) {
+  const int slot = px.seq & 1;
+  if ((threadIdx.x & 31) == 0) {
+    px.slots[2 * slot + px.w] = mine;
+    ptx::mbar_arrive(px.bar);
+  }
+  ok = ptx::mbar_wait(px.bar, px.seq & 1, px.status, kTimeoutCode) && ok;
+  const uint4 r = px.slots[2 * slot + (px.w ^ 1)];
+  ++px.seq;
+  return r;
 }
 
 __device__ __forceinline__ void fma_x2(float& d0, float& d1, float a0, float a1, uint64_t bb, float c0, float c1) {
@@ -439,7 +467,9 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
                                               uint32_t tscratch, uint32_t& lo_dirty, RowState& st,
                                               float (&lam)[4], WarpCounters& wc, unsigned long long (&cks)[2],
                                               int dump_row0, int row0, long long* ph, uint64_t* pv_bar,
-                                              uint32_t pv_parity, bool pv_wait, int* status, bool& ok, const unsigned char* q_quad) {
+                                              uint32_t pv_parity, bool pv_wait, int* status, bool& ok, const unsigned char* q_quad,
+                                              PairX& px) {
+  constexpr bool PAIR = (VAR == 5);
   const int lane = threadIdx.x & 31;
   const int qa = lane >> 2, th_own = lane & 3;
   const double scale_d = (double)P.scale;
@@ -490,7 +520,7 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
     bool act = true;
     if (!FULL) {
       const int s0 = g.i0 + 16 * th;
-      act = s0 < g.n && (!g.causal || s0 <= min(g.j0 + g.bq - 1, g.n - 1)) && (g.window == 0 || g.j0 - (s0 + 15) < g.window);
+      act = s0 < g.n && (!g.causal || s0 <= min(g.gj0 + g.gbq - 1, g.n - 1)) && (g.window == 0 || g.gj0 - (s0 + 15) < g.window);
     }
     actmask |= (uint32_t)act << th;
   }
@@ -507,6 +537,12 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
   float T[4];
 #pragma unroll
   for (int th = 0; th < 4; ++th) T[th] = __shfl_sync(kFull, tl, th);
+  if constexpr (PAIR) {
+    const uint4 o = pair_exchange(px, make_uint4(__float_as_uint(T[0]), __float_as_uint(T[1]), __float_as_uint(T[2]),
+                                                 __float_as_uint(T[3])), ok);
+    T[0] = fmaxf(T[0], __uint_as_float(o.x)); T[1] = fmaxf(T[1], __uint_as_float(o.y));
+    T[2] = fmaxf(T[2], __uint_as_float(o.z)); T[3] = fmaxf(T[3], __uint_as_float(o.w));
+  }
   uint32_t order = 0;   // 2 bits per rank: the sub-block visited at that rank
 #pragma unroll
   for (int th = 0; th < 4; ++th) {
@@ -539,6 +575,7 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
           }
       }
       fail = __any_sync(kFull, f);
+      if constexpr (PAIR) fail |= pair_exchange(px, make_uint4(fail, 0, 0, 0), ok).x != 0;
     }
     if (!fail) continue;
     Theta |= 1u << th;
@@ -688,7 +725,8 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
               uint32_t yb = (ya[c] >> (8 * (u + v))) & 0xffu;
               if (yb == 0x80u) yb = 0;                       // -0 is stored as +0
               const uint32_t ebb = own8 ? enc_exp8(ee[v]) : 0xffu;
-              const uint64_t idx = (uint64_t)((16 * th_own + b + v) * kBQ + 4 * qa + a) << 8;
+              const uint64_t idx = PAIR ? (uint64_t)((16 * th_own + b + v) * 64 + 32 * px.w + 4 * qa + a) << 8
+                                        : (uint64_t)((16 * th_own + b + v) * kBQ + 4 * qa + a) << 8;
               cks[0] += mix64(idx | yb);
               cks[1] += mix64(idx | ebb);
               if (dump_row0 >= 0) {
@@ -759,6 +797,7 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
     for (int a = 0; a < 4; ++a)
       need2 |= !(r8free[a] <= __dmul_rn((double)P.tau * 0.999999998, (double)omh[a]));
     need2 = __any_sync(kFull, need2);
+    if constexpr (PAIR) need2 |= pair_exchange(px, make_uint4(need2, 0, 0, 0), ok).x != 0;
   }
   if (need2) {
     double xi[4] = {0.0, 0.0, 0.0, 0.0};
@@ -805,6 +844,7 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
       }
     }
     feas = __reduce_and_sync(kFull, feas);
+    if constexpr (PAIR) feas &= pair_exchange(px, make_uint4(feas, 0, 0, 0), ok).x;
     int best = 5;   // smallest recompute set, then smallest bitmask, among subsets of the free ones
 #pragma unroll 1
     for (uint32_t r = 0; r < 16; ++r) {
@@ -865,11 +905,13 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
   }
   lo_dirty = hi16;
 
-  if (__any_sync(kFull, big)) wc.bigrow++;
-  wc.active += nact;
-  wc.s1 += __popc(Theta);
-  wc.s2 += __popc(Rset);
-  {
+  bool bigw = __any_sync(kFull, big);
+  if constexpr (PAIR) bigw |= pair_exchange(px, make_uint4(bigw, 0, 0, 0), ok).x != 0;
+  if (!PAIR || px.w == 0) {   // per-group counters: once per group
+    if (bigw) wc.bigrow++;
+    wc.active += nact;
+    wc.s1 += __popc(Theta);
+    wc.s2 += __popc(Rset);
     const int pc = __popc(hi16);
 #pragma unroll
     for (int i = 0; i < 5; ++i) wc.hist[i] += (pc == i);
@@ -880,7 +922,7 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
 
 // VAR 1: the per-step reading of the 16-bit accumulation (mode LAMP_H16_SEQ); VAR 2: stochastic rounding in
 // the first pass (mode LAMP_SR_E4M3); VAR 3: LAMP_FORCE_16BIT without debug outputs, the first pass skipped;
-// VAR 4: groups of 16 instead of 32 rows (group_rows = 16).  Kernels of their own, so that the default one (VAR 0) carries nothing
+// VAR 4: groups of 16 instead of 32 rows (group_rows = 16); VAR 5: groups of 64 rows, two warps vote together.  Kernels of their own, so that the default one (VAR 0) carries nothing
 // of them (code that never ran still cost it 2.5 % through register allocation).
 template <int D, bool DUMP, int VAR>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -937,6 +979,8 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
       ptx::mbar_init(&bars[kPvDone0 + i], 1);
     }
     for (int i = 0; i < 8 * kSlots; ++i) ptx::mbar_init(&bars[kSlotFull0 + i], 1);
+    ptx::mbar_init(&bars[kPairBar0], 2);
+    ptx::mbar_init(&bars[kPairBar0 + 1], 2);
     ptx::fence_barrier_init();
     for (int i = 0; i < 8; ++i) lomask[i] = 0;
   }
@@ -1160,6 +1204,13 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
     const __nv_bfloat16* kg = P.k + b * P.ks[0] + hk * P.ks[1];
     double* dscr = dscr_all + grp * 384;
     const unsigned char* q_quad = VAR == 1 ? qs + (QF32 ? 4 : 2) * (grp * kBQ + 4 * qa) : nullptr;
+    constexpr bool PAIR = (VAR == 5);            // groups of 64 rows: warps 2p and 2p+1 decide together
+    constexpr int gbq = PAIR ? 64 : bq;
+    const int gj0 = PAIR ? m0 + (grp >> 1) * 64 : j0;
+    PairX px;
+    px.slots = reinterpret_cast<uint4*>(smem + L::kPairX) + 4 * (grp >> 1);
+    px.bar = &bars[kPairBar0 + (grp >> 1)];
+    px.seq = 0; px.w = grp & 1; px.status = status;
     const uint32_t tlane = tbase + ((uint32_t)(grp * 32) << 16);
     const uint32_t tscr = tlane + kColScr, tq = tlane + kColQ, tring = tlane + kColRing;
     {
@@ -1198,9 +1249,10 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
     for (int n = 0; n < T && ok; ++n) {
       const int t = t_begin + n, i0 = t * kTK;
       TileGeom g;
-      g.i0 = i0; g.j0 = j0; g.causal = P.causal; g.window = P.window; g.n = P.seqlen; g.bq = bq;
-      const bool any = j0 < P.seqlen && (!P.causal || i0 <= min(j0 + bq - 1, P.seqlen - 1)) &&
-                       (P.window == 0 || j0 - (i0 + 63) < P.window);
+      g.i0 = i0; g.j0 = j0; g.causal = P.causal; g.window = P.window; g.n = P.seqlen; g.bq = bq; g.gj0 = gj0; g.gbq = gbq;
+      // (with 64-row groups a warp also walks the tiles only its partner's rows see: the votes need both)
+      const bool any = gj0 < P.seqlen && (!P.causal || i0 <= min(gj0 + gbq - 1, P.seqlen - 1)) &&
+                       (P.window == 0 || gj0 - (i0 + 63) < P.window);
       const bool full = bq == kBQ && j0 + 31 < P.seqlen && i0 + 63 < P.seqlen && (!P.causal || i0 + 63 <= j0) &&
                         (P.window == 0 || (j0 + 31) - i0 < P.window);
       float lam[4] = {1.0f, 1.0f, 1.0f, 1.0f};
@@ -1229,11 +1281,11 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
         if (full)
           flag = lamp_post<D, true, DUMP, VAR>(P, g, yw, ktile, P.ks[2], tq, lut, dscr, phi, plo, tscr, lo_dirty,
                                           st, lam, wc, cks, dump0, grp * kBQ, ph, &bars[kPvDone0 + grp], (n - 1) & 1, n > 0,
-                                          status, ok, q_quad);
+                                          status, ok, q_quad, px);
         else
           flag = lamp_post<D, false, DUMP, VAR>(P, g, yw, ktile, P.ks[2], tq, lut, dscr, phi, plo, tscr, lo_dirty,
                                            st, lam, wc, cks, dump0, grp * kBQ, ph, &bars[kPvDone0 + grp], (n - 1) & 1, n > 0,
-                                           status, ok, q_quad);
+                                           status, ok, q_quad, px);
       } else {
         // no visible pair for this group: its rows of the P tile are zero (once the previous
         // P V product has read them)
@@ -1276,15 +1328,18 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
       if (lane == 0) ptx::mbar_arrive(&bars[kPReady0 + grp]);
       LAMP_TOC(7, t_r);
 
-      const int64_t gt = (((int64_t)b * P.heads_q + h) * ((P.seqlen + bq - 1) / bq) + (j0 / bq)) * ntk + t;
-      if (lane == 0 && P.flag_mask && j0 < P.seqlen) P.flag_mask[gt] = (uint8_t)flag;
-      if (DUMP && P.dbg_checksums && j0 < P.seqlen) {
+      const int64_t gt = (((int64_t)b * P.heads_q + h) * ((P.seqlen + gbq - 1) / gbq) + (gj0 / gbq)) * ntk + t;
+      if (lane == 0 && P.flag_mask && gj0 < P.seqlen && (!PAIR || px.w == 0)) P.flag_mask[gt] = (uint8_t)flag;
+      if (DUMP && P.dbg_checksums && gj0 < P.seqlen) {
 #pragma unroll
         for (int s = 16; s > 0; s >>= 1) {
           cks[0] += __shfl_xor_sync(kFull, cks[0], s);
           cks[1] += __shfl_xor_sync(kFull, cks[1], s);
         }
-        if (lane == 0) { P.dbg_checksums[2 * gt] = cks[0]; P.dbg_checksums[2 * gt + 1] = cks[1]; }
+        if (lane == 0) {
+          if (PAIR) { atomicAdd(&P.dbg_checksums[2 * gt], cks[0]); atomicAdd(&P.dbg_checksums[2 * gt + 1], cks[1]); }   // two warps, one entry
+          else { P.dbg_checksums[2 * gt] = cks[0]; P.dbg_checksums[2 * gt + 1] = cks[1]; }
+        }
       }
     }
 

@@ -97,23 +97,23 @@ def test_ragged_sequence_lengths(N, causal, window, D, flags):
     compare_dense_bytes(gpu, ref, 1, 1)
 
 
+@pytest.mark.parametrize("bq", [16, 64])
 @pytest.mark.parametrize("N,causal,window,D,flags,tau", [(512, True, 0, 128, 0, 0.5), (333, True, 0, 128, 0, 0.125),
                                                          (384, False, 0, 128, 0, 0.5), (300, True, 100, 128, 0, 0.5),
                                                          (256, True, 0, 256, 0, 0.5), (200, True, 0, 128, oracle.FORCE_16BIT, 0.5),
-                                                         (200, True, 0, 128, oracle.COMPACT_BRANCH, 0.25), (48, True, 0, 128, 0, 0.5)])
-def test_group_of_sixteen_rows(N, causal, window, D, flags, tau):
-    """b_q = 16: sixteen query rows decide together instead of a warp's thirty-two (the other instance of the group
-    size the paper leaves open); the flag mask has twice as many groups."""
+                                                         (200, True, 0, 128, oracle.COMPACT_BRANCH, 0.25), (48, True, 0, 128, 0, 0.5),
+                                                         (96, True, 0, 128, oracle.NO_STAGE1, 0.125)])
+def test_other_group_sizes(N, causal, window, D, flags, tau, bq):
+    """b_q = 16 and 64: sixteen rows, or two warps' sixty-four, decide together instead of a warp's thirty-two (the
+    other instances of the group size the paper leaves open); the flag mask has N/16 resp. N/64 groups."""
     cfg = li.CONFIGS[1 if D == 128 else 3]
     q, k, v = li.make_qkv(cfg, B=1, Hq=2, Hkv=1, N=N, seed=90 + N)
     sc = li.softmax_scale(cfg.D)
-    ref = oracle.run_all(q, k, v, scale=sc, causal=causal, window=window, flags=flags, tau=tau, group_rows=16, dumps=True)
-    gpu = run_gpu(q, k, v, scale=sc, causal=causal, window=window, flags=flags, threshold=tau, group_rows=16, dump=(0, 1))
-    assert gpu["flags"].shape[2] == (N + 15) // 16
-    compare_units(gpu, ref, check_stats=True, label=f"bq16 N={N} flags={flags}", bq=16)
-    compare_dense_bytes(gpu, ref, 0, 1, bq=16)
-    ref32 = oracle.run_all(q, k, v, scale=sc, causal=causal, window=window, flags=flags, tau=tau)
-    assert flags or ref32.stats["stage1_flagged"] >= ref.stats["stage1_flagged"] // 2
+    ref = oracle.run_all(q, k, v, scale=sc, causal=causal, window=window, flags=flags, tau=tau, group_rows=bq, dumps=True)
+    gpu = run_gpu(q, k, v, scale=sc, causal=causal, window=window, flags=flags, threshold=tau, group_rows=bq, dump=(0, 1))
+    assert gpu["flags"].shape[2] == (N + bq - 1) // bq
+    compare_units(gpu, ref, check_stats=True, label=f"bq={bq} N={N} flags={flags}", bq=bq)
+    compare_dense_bytes(gpu, ref, 0, 1, bq=bq)
 
 
 @pytest.mark.parametrize("mult", [0.5, 4.0, 8.0])
