@@ -150,6 +150,10 @@ size_t lamp_attn_workspace_bytes(const lamp_attn_params* p);
  *   cuda_stream a cudaStream_t (NULL = the default stream)
  * Inputs must be finite.  Logits beyond +-448 saturate (counted, not an error).  batch = 0 or seqlen = 0 is an
  * empty problem: LAMP_OK, nothing is enqueued and no pointer is looked at.
+ * The call enqueues a few memsets and one kernel on the stream and nothing else, so after one call on the
+ * device outside any capture (the one-time set-up) it may be recorded in a CUDA graph; a replay reads and
+ * writes the buffers given at capture.  The outputs are a deterministic function of the inputs: repeated
+ * calls give the same bytes.
  * Errors: LAMP_ERR_INVALID_ARG, LAMP_ERR_UNSUPPORTED_SHAPE, LAMP_ERR_UNSUPPORTED_DEVICE,
  * LAMP_ERR_CUDA; nothing is enqueued when an error is returned. */
 int lamp_attn_fwd(const void* q, const void* k, const void* v, void* out, float* lse,

@@ -254,6 +254,41 @@ def test_strided_inputs_and_bf16_output():
     assert torch.equal(c["out"], b["out"].to(torch.bfloat16))
 
 
+def test_repeatable_capturable_and_safe_on_two_streams():
+    """Same inputs, same bytes: call after call, from a replayed CUDA graph, and from two streams at once."""
+    import paper_2609_39361_b200 as lamp
+    dev = torch.device("cuda:0")
+    cfg = li.CONFIGS[1]
+    sc = li.softmax_scale(cfg.D)
+    qa, ka, va = [t.to(dev) for t in li.make_qkv(cfg, Hq=4, Hkv=2, N=1100, seed=31)]
+    qb, kb, vb = [t.to(dev) for t in li.make_qkv(cfg, Hq=4, Hkv=2, N=1100, seed=32)]
+    same = lambda x, y: all(torch.equal(x[n], y[n]) for n in ("out", "lse", "flags"))
+    ra, rb = lamp.forward(qa, ka, va, scale=sc), lamp.forward(qb, kb, vb, scale=sc)
+    assert same(ra, lamp.forward(qa, ka, va, scale=sc))
+    assert not torch.equal(ra["out"], rb["out"])
+    # graph: capture on inputs A, replay, then overwrite the captured input buffers with B and replay again
+    qg, kg, vg = qa.clone(), ka.clone(), va.clone()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        rg = lamp.forward(qg, kg, vg, scale=sc)
+    g.replay(); torch.cuda.synchronize()
+    assert same(rg, ra)
+    qg.copy_(qb); kg.copy_(kb); vg.copy_(vb)
+    g.replay(); torch.cuda.synchronize()
+    assert same(rg, rb)
+    # two streams, kernels free to overlap
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(s1):
+        r1 = [lamp.forward(qa, ka, va, scale=sc) for _ in range(3)]
+    with torch.cuda.stream(s2):
+        r2 = [lamp.forward(qb, kb, vb, scale=sc) for _ in range(3)]
+    torch.cuda.synchronize()
+    assert all(same(r, ra) for r in r1) and all(same(r, rb) for r in r2)
+    assert lamp.lamp_attn_get_stats()["device_status"] == 0
+
+
 def test_empty_problems_are_accepted():
     import paper_2609_39361_b200 as lamp
     dev = torch.device("cuda:0")
