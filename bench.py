@@ -295,10 +295,12 @@ def main():
     hl = torch.empty(B, Hq, N, dtype=torch.float32).pin_memory()
     hf = torch.empty(B, Hq, N // GR, N // 64, dtype=torch.uint8).pin_memory()
 
+    ws = torch.empty(lamp.lamp_attn_host_workspace_bytes(p), device=dev, dtype=torch.uint8)
+
     def e2e_step():
-        dq.copy_(hq, non_blocking=True); dk.copy_(hk, non_blocking=True); dv.copy_(hv, non_blocking=True)
-        step()
-        ho.copy_(out, non_blocking=True); hl.copy_(lse, non_blocking=True); hf.copy_(fm, non_blocking=True)
+        # the library's host-memory call: Q, K, V from page-locked host memory, O, lse and the flag mask back to it,
+        # the copies of one range of heads overlapped with the kernel of another
+        lamp.lamp_attn_fwd_host(hq, hk, hv, ho, hl, hf, p, ws)
 
     e2e_step()
     barrier()

@@ -160,6 +160,30 @@ int lamp_attn_fwd(const void* q, const void* k, const void* v, void* out, float*
                   uint8_t* flag_mask, const lamp_attn_params* p, void* workspace,
                   size_t workspace_bytes, void* cuda_stream);
 
+/* The same forward pass for tensors that live in HOST memory.
+ * (The paper has no counterpart of this call; it is a service of this library.)
+ *   q_host, k_host, v_host   host, bf16, contiguous [batch, heads, seqlen, head_dim]; read
+ *   out_host                 host, bf16 (fp32 with LAMP_OUT_FP32), contiguous; written
+ *   lse_host, flag_mask_host host, contiguous, layouts as for lamp_attn_fwd; written; may be NULL
+ *   p          host; sizes, thresholds, flags and group_rows as for lamp_attn_fwd; the stride fields are not
+ *              read (host tensors are contiguous); LAMP_SR_E4M3 and the dbg_* outputs are not available here
+ *   workspace  device, 256-byte aligned, at least lamp_attn_host_workspace_bytes(p) bytes (the size of all six
+ *              tensors): the library allocates no device memory here either
+ * The (batch, kv head) pairs are independent problems (Sec. 3.3: the heads do not interact), so the call cuts them
+ * into up to 8 ranges and overlaps the host-to-device copy of one range and the device-to-host copy of another
+ * with the kernel of a third, on two streams of its own that are ordered with cuda_stream by events: the call
+ * is asynchronous, work queued on cuda_stream before it has finished before the workspace is touched, and work
+ * queued on cuda_stream after it (or a synchronisation of that stream) sees the complete results in host
+ * memory.  Use page-locked host memory: pageable memory is correct but the copies then block the calling thread
+ * and do not overlap.  Results are byte-identical to lamp_attn_fwd on the same data; the counters of
+ * lamp_attn_get_stats cover the whole call.  Host threads calling this on one device are serialised.
+ * Errors as for lamp_attn_fwd; a LAMP_ERR_CUDA that comes from an enqueue in mid-call leaves part of the
+ * work queued. */
+size_t lamp_attn_host_workspace_bytes(const lamp_attn_params* p);
+int lamp_attn_fwd_host(const void* q_host, const void* k_host, const void* v_host, void* out_host,
+                       float* lse_host, uint8_t* flag_mask_host, const lamp_attn_params* p,
+                       void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Forward pass plus a fingerprint of its low-precision stage, for callers that cannot allocate.
  * (The paper has no counterpart of this call; it is a service of this library.)
  *

@@ -8,5 +8,5 @@ from .binding import (  # noqa: F401
     LAMP_COMPACT_BRANCH, LAMP_FORCE_16BIT, LAMP_H16_SEQ, LAMP_SR_E4M3, LAMP_FORCE_8BIT, LAMP_NO_STAGE1, LAMP_OUT_FP32, LampAttnError,
     LampAttnParams, LampAttnStats, lamp_attn_contiguous_strides, lamp_attn_default_params,
     lamp_attn_fwd, lamp_attn_fwd_digest, lamp_attn_debug_round_e4m3, lamp_attn_debug_exp16, lamp_attn_get_stats, LAMP_DIGEST_MAX_PAIRS, lamp_attn_last_cuda_error, lamp_attn_strerror,
-    lamp_attn_workspace_bytes, library, forward,
+    lamp_attn_workspace_bytes, lamp_attn_host_workspace_bytes, lamp_attn_fwd_host, library, forward,
 )

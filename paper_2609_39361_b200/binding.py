@@ -10,7 +10,7 @@ _LIB_PATH = os.path.join(_HERE, "liblamp_attn.so")
 LAMP_FORCE_16BIT, LAMP_FORCE_8BIT, LAMP_NO_STAGE1, LAMP_OUT_FP32, LAMP_COMPACT_BRANCH, LAMP_H16_SEQ, LAMP_SR_E4M3 = 1, 2, 4, 8, 16, 32, 64
 
 EXPORTS = ("lamp_attn_default_params", "lamp_attn_contiguous_strides", "lamp_attn_workspace_bytes",
-           "lamp_attn_fwd", "lamp_attn_fwd_digest", "lamp_attn_debug_round_e4m3", "lamp_attn_debug_exp16", "lamp_attn_get_stats", "lamp_attn_last_cuda_error", "lamp_attn_strerror")
+           "lamp_attn_fwd", "lamp_attn_host_workspace_bytes", "lamp_attn_fwd_host", "lamp_attn_fwd_digest", "lamp_attn_debug_round_e4m3", "lamp_attn_debug_exp16", "lamp_attn_get_stats", "lamp_attn_last_cuda_error", "lamp_attn_strerror")
 
 
 class LampAttnError(RuntimeError):
@@ -62,6 +62,9 @@ def library():
         L.lamp_attn_workspace_bytes.restype = C.c_size_t; L.lamp_attn_workspace_bytes.argtypes = [PP]
         L.lamp_attn_fwd.restype = C.c_int
         L.lamp_attn_fwd.argtypes = [C.c_void_p] * 6 + [PP, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.lamp_attn_host_workspace_bytes.restype = C.c_size_t; L.lamp_attn_host_workspace_bytes.argtypes = [PP]
+        L.lamp_attn_fwd_host.restype = C.c_int
+        L.lamp_attn_fwd_host.argtypes = [C.c_void_p] * 6 + [PP, C.c_void_p, C.c_size_t, C.c_void_p]
         L.lamp_attn_fwd_digest.restype = C.c_int
         L.lamp_attn_fwd_digest.argtypes = [C.c_void_p] * 6 + [PP, C.c_void_p, C.c_void_p]
         L.lamp_attn_debug_round_e4m3.restype = C.c_int
@@ -116,6 +119,23 @@ def lamp_attn_fwd(q, k, v, out, lse, flag_mask, p: LampAttnParams, workspace=Non
     rc = library().lamp_attn_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), _ptr(flag_mask),
                                  C.byref(p), _ptr(workspace), ws_bytes, C.c_void_p(s))
     _check(rc, "lamp_attn_fwd")
+
+
+def lamp_attn_host_workspace_bytes(p: LampAttnParams) -> int:
+    return int(library().lamp_attn_host_workspace_bytes(C.byref(p)))
+
+
+def lamp_attn_fwd_host(q, k, v, out, lse, flag_mask, p: LampAttnParams, workspace, stream=None) -> None:
+    """q, k, v, out, lse, flag_mask: contiguous CPU tensors (page-locked for overlapped copies; lse and flag_mask
+    may be None); workspace: CUDA uint8 tensor of at least lamp_attn_host_workspace_bytes(p) bytes.
+    Asynchronous: synchronise the stream before reading the outputs."""
+    import torch
+    for t in (q, k, v, out, lse, flag_mask):
+        assert t is None or (not t.is_cuda and t.is_contiguous())
+    s = torch.cuda.current_stream().cuda_stream if stream is None else stream
+    rc = library().lamp_attn_fwd_host(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), _ptr(flag_mask), C.byref(p),
+                                      _ptr(workspace), workspace.numel() * workspace.element_size(), C.c_void_p(s))
+    _check(rc, "lamp_attn_fwd_host")
 
 
 def lamp_attn_debug_round_e4m3(x, out=None, stream=None):

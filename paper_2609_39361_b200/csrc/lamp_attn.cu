@@ -4,6 +4,8 @@
 #include <math.h>
 #include <string.h>
 
+#include <mutex>
+
 #include "lamp_common.cuh"
 #include "lamp_fwd_sm100.cuh"
 
@@ -57,6 +59,8 @@ struct DeviceInit {
   bool ready[64] = {};
 };
 static DeviceInit g_init;
+
+constexpr int kHostChunks = 8;   // ranges a host-memory call is cut into (lamp_attn_fwd_host)
 
 static int ensure_device(int* dev_out) {
   int dev = 0;
@@ -185,6 +189,7 @@ static int check_params(const void* q, const void* k, const void* v, void* out,
     return LAMP_ERR_INVALID_ARG;
   if (p->head_dim != 128 && p->head_dim != 256) return LAMP_ERR_UNSUPPORTED_SHAPE;
   if (p->batch > 65535 || p->heads_q > 65535) return LAMP_ERR_UNSUPPORTED_SHAPE;
+  if ((long long)((p->seqlen + 63) / 64) * p->heads_q * p->batch > 0x7fffffffLL) return LAMP_ERR_UNSUPPORTED_SHAPE;   // blocks of one launch
   const int D = p->head_dim;
   if (!strides_ok(p->q_strides, D) || !strides_ok(p->k_strides, D) ||
       !strides_ok(p->v_strides, D) || !strides_ok(p->o_strides, D))
@@ -193,19 +198,19 @@ static int check_params(const void* q, const void* k, const void* v, void* out,
   return LAMP_OK;
 }
 
-int lamp_attn_fwd(const void* q, const void* k, const void* v, void* out, float* lse,
-                  uint8_t* flag_mask, const lamp_attn_params* p, void* workspace,
-                  size_t workspace_bytes, void* cuda_stream) {
-  (void)workspace; (void)workspace_bytes;
-  // an empty problem (no batch entries or no tokens) is valid and enqueues nothing
-  if (p && (p->batch == 0 || p->seqlen == 0) && p->batch >= 0 && p->seqlen >= 0 && p->heads_q > 0 && p->heads_kv > 0)
-    return LAMP_OK;
+static bool empty_problem(const lamp_attn_params* p) {
+  return p && (p->batch == 0 || p->seqlen == 0) && p->batch >= 0 && p->seqlen >= 0 && p->heads_q > 0 && p->heads_kv > 0;
+}
+
+// Checks, the memsets of the outputs that need one, and the launch.  clear_stats: start the device counters
+// from zero (a call that is split into several launches clears them once).
+static int fwd_enqueue(const void* q, const void* k, const void* v, void* out, float* lse,
+                       uint8_t* flag_mask, const lamp_attn_params* p, cudaStream_t stream, bool clear_stats) {
   int rc = check_params(q, k, v, out, p);
   if (rc) return rc;
   int dev;
   rc = ensure_device(&dev);
   if (rc) return rc;
-  cudaStream_t stream = (cudaStream_t)cuda_stream;
 
   KernelParams P;
   P.q = (const __nv_bfloat16*)q; P.k = (const __nv_bfloat16*)k; P.v = (const __nv_bfloat16*)v;
@@ -225,8 +230,10 @@ int lamp_attn_fwd(const void* q, const void* k, const void* v, void* out, float*
   void* stats_ptr = nullptr;
   cudaError_t e = cudaGetSymbolAddress(&stats_ptr, g_stats);
   if (e != cudaSuccess) return cuda_fail(e);
-  e = cudaMemsetAsync(stats_ptr, 0, sizeof(DeviceStats), stream);
-  if (e != cudaSuccess) return cuda_fail(e);
+  if (clear_stats) {
+    e = cudaMemsetAsync(stats_ptr, 0, sizeof(DeviceStats), stream);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
 
   const int bq = p->group_rows ? p->group_rows : kBQ;
   const size_t ngt = (size_t)p->batch * p->heads_q * ((p->seqlen + bq - 1) / bq) * ((p->seqlen + kTK - 1) / kTK);
@@ -248,7 +255,8 @@ int lamp_attn_fwd(const void* q, const void* k, const void* v, void* out, float*
   if (rc) return rc;
   const bool dump = p->dbg_y8 || p->dbg_e8 || p->dbg_checksums;
   const int cta_rows = bq == 16 ? 64 : 128;
-  dim3 grid((p->seqlen + cta_rows - 1) / cta_rows, p->heads_q, p->batch), block(kThreads);
+  // one block per (query tile, head, batch entry), the tile index slowest: see the kernel's block mapping
+  dim3 grid((unsigned)((p->seqlen + cta_rows - 1) / cta_rows) * p->heads_q * p->batch), block(kThreads);
   const uint2* lutp = (const uint2*)lut_ptr;
   DeviceStats* dsp = (DeviceStats*)stats_ptr;
 #define LAMP_LAUNCH(D_, DUMP_, VAR_) \
@@ -277,6 +285,15 @@ int lamp_attn_fwd(const void* q, const void* k, const void* v, void* out, float*
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
   return LAMP_OK;
+}
+
+int lamp_attn_fwd(const void* q, const void* k, const void* v, void* out, float* lse,
+                  uint8_t* flag_mask, const lamp_attn_params* p, void* workspace,
+                  size_t workspace_bytes, void* cuda_stream) {
+  (void)workspace; (void)workspace_bytes;
+  // an empty problem (no batch entries or no tokens) is valid and enqueues nothing
+  if (empty_problem(p)) return LAMP_OK;
+  return fwd_enqueue(q, k, v, out, lse, flag_mask, p, (cudaStream_t)cuda_stream, true);
 }
 
 }  // extern "C"
@@ -361,6 +378,128 @@ int lamp_attn_fwd_digest(const void* q, const void* k, const void* v, void* out,
                                                  (unsigned long long*)digest);
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
+  return LAMP_OK;
+}
+
+// ---- host-memory entry point: staged through a caller-provided device workspace, copies overlapped ----
+// The (batch, kv head) pairs are independent problems, so the call is cut into up to kHostChunks ranges of
+// them: range i is copied in on one internal stream, computed on the caller's stream and copied out on a second
+// internal stream, ordered by events only; while range i computes, range i+1 arrives and range i-1 leaves.
+struct HostPipe {
+  cudaStream_t in = nullptr, out = nullptr;
+  cudaEvent_t start = nullptr, done = nullptr, arrived[kHostChunks] = {}, computed[kHostChunks] = {};
+  bool ready = false;
+};
+static HostPipe g_pipe[64];
+static std::mutex g_pipe_mutex;
+
+struct HostLayout {
+  size_t q, k, v, o, lse, fm, total;        // offsets into the workspace
+  size_t qh, kh, oh, lh, fh;                // bytes per query head (q, out, lse, flags) / per kv head (k, v)
+};
+static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+static HostLayout host_layout(const lamp_attn_params* p) {
+  HostLayout L;
+  const size_t N = p->seqlen, D = p->head_dim, bq = p->group_rows ? p->group_rows : kBQ;
+  const size_t HQ = (size_t)p->batch * p->heads_q, HK = (size_t)p->batch * p->heads_kv;
+  L.qh = N * D * 2; L.kh = N * D * 2; L.oh = N * D * ((p->flags & LAMP_OUT_FP32) ? 4 : 2);
+  L.lh = N * 4; L.fh = ((N + bq - 1) / bq) * ((N + kTK - 1) / kTK);
+  L.q = 0; L.k = L.q + align256(HQ * L.qh); L.v = L.k + align256(HK * L.kh); L.o = L.v + align256(HK * L.kh);
+  L.lse = L.o + align256(HQ * L.oh); L.fm = L.lse + align256(HQ * L.lh); L.total = L.fm + align256(HQ * L.fh);
+  return L;
+}
+
+static bool host_params_ok(const lamp_attn_params* p) {
+  return p && p->batch >= 0 && p->seqlen >= 0 && p->heads_q > 0 && p->heads_kv > 0 && p->heads_q % p->heads_kv == 0 &&
+         (p->head_dim == 128 || p->head_dim == 256) &&
+         (p->group_rows == 0 || p->group_rows == 16 || p->group_rows == 32 || p->group_rows == 64);
+}
+
+size_t lamp_attn_host_workspace_bytes(const lamp_attn_params* p) {
+  if (!host_params_ok(p)) return 0;
+  return host_layout(p).total;
+}
+
+int lamp_attn_fwd_host(const void* q_host, const void* k_host, const void* v_host, void* out_host, float* lse_host,
+                       uint8_t* flag_mask_host, const lamp_attn_params* p, void* workspace, size_t workspace_bytes,
+                       void* cuda_stream) {
+  if (!host_params_ok(p)) return p && p->head_dim != 128 && p->head_dim != 256 && p->head_dim > 0
+                                     ? LAMP_ERR_UNSUPPORTED_SHAPE : LAMP_ERR_INVALID_ARG;
+  if (empty_problem(p)) return LAMP_OK;
+  if (!q_host || !k_host || !v_host || !out_host) return LAMP_ERR_INVALID_ARG;
+  if (p->dbg_y8 || p->dbg_e8 || p->dbg_checksums || (p->flags & LAMP_SR_E4M3)) return LAMP_ERR_INVALID_ARG;
+  const HostLayout L = host_layout(p);
+  if (!workspace || workspace_bytes < L.total || ((uintptr_t)workspace & 255)) return LAMP_ERR_INVALID_ARG;
+  const int rep = p->heads_q / p->heads_kv;
+  const long long U = (long long)p->batch * p->heads_kv;          // independent (batch, kv head) problems
+  const int chunks = (int)(U < kHostChunks ? U : kHostChunks);
+  if ((U + chunks - 1) / chunks * rep > 65535) return LAMP_ERR_UNSUPPORTED_SHAPE;
+
+  // each range runs as one batch entry with (range length) kv heads over contiguous tensors
+  lamp_attn_params pp = *p;
+  pp.batch = 1;
+  pp.dbg_batch = pp.dbg_head = 0;
+  char* ws = (char*)workspace;
+  // every argument check of the launches, before anything is enqueued
+  {
+    pp.heads_kv = 1; pp.heads_q = rep;
+    lamp_attn_contiguous_strides(&pp);
+    const int rc = check_params(ws + L.q, ws + L.k, ws + L.v, ws + L.o, &pp);
+    if (rc) return rc;
+  }
+  int dev;
+  int rc = ensure_device(&dev);
+  if (rc) return rc;
+  if (dev < 0 || dev >= 64) return LAMP_ERR_UNSUPPORTED_DEVICE;
+  std::lock_guard<std::mutex> lock(g_pipe_mutex);
+  HostPipe& hp = g_pipe[dev];
+  cudaError_t e;
+  if (!hp.ready) {
+    if ((e = cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaEventCreateWithFlags(&hp.done, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+    for (int i = 0; i < kHostChunks; ++i) {
+      if ((e = cudaEventCreateWithFlags(&hp.arrived[i], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+      if ((e = cudaEventCreateWithFlags(&hp.computed[i], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+    }
+    hp.ready = true;
+  }
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+#define LAMP_TRY(call) do { e = (call); if (e != cudaSuccess) return cuda_fail(e); } while (0)
+  // the copies may not overtake work already queued on the caller's stream (it may still use the workspace)
+  LAMP_TRY(cudaEventRecord(hp.start, stream));
+  LAMP_TRY(cudaStreamWaitEvent(hp.in, hp.start, 0));
+  LAMP_TRY(cudaStreamWaitEvent(hp.out, hp.start, 0));
+  void* stats_ptr = nullptr;
+  LAMP_TRY(cudaGetSymbolAddress(&stats_ptr, g_stats));
+  LAMP_TRY(cudaMemsetAsync(stats_ptr, 0, sizeof(DeviceStats), stream));
+  for (int c = 0; c < chunks; ++c) {
+    const size_t u0 = (size_t)(U * c / chunks), nu = (size_t)(U * (c + 1) / chunks) - u0;
+    const size_t h0 = u0 * rep, nh = nu * rep;
+    LAMP_TRY(cudaMemcpyAsync(ws + L.q + h0 * L.qh, (const char*)q_host + h0 * L.qh, nh * L.qh, cudaMemcpyHostToDevice, hp.in));
+    LAMP_TRY(cudaMemcpyAsync(ws + L.k + u0 * L.kh, (const char*)k_host + u0 * L.kh, nu * L.kh, cudaMemcpyHostToDevice, hp.in));
+    LAMP_TRY(cudaMemcpyAsync(ws + L.v + u0 * L.kh, (const char*)v_host + u0 * L.kh, nu * L.kh, cudaMemcpyHostToDevice, hp.in));
+    LAMP_TRY(cudaEventRecord(hp.arrived[c], hp.in));
+    LAMP_TRY(cudaStreamWaitEvent(stream, hp.arrived[c], 0));
+    pp.heads_kv = (int)nu; pp.heads_q = (int)nh;
+    lamp_attn_contiguous_strides(&pp);
+    rc = fwd_enqueue(ws + L.q + h0 * L.qh, ws + L.k + u0 * L.kh, ws + L.v + u0 * L.kh, ws + L.o + h0 * L.oh,
+                     lse_host ? (float*)(ws + L.lse + h0 * L.lh) : nullptr,
+                     flag_mask_host ? (uint8_t*)(ws + L.fm + h0 * L.fh) : nullptr, &pp, stream, false);
+    if (rc) return rc;
+    LAMP_TRY(cudaEventRecord(hp.computed[c], stream));
+    LAMP_TRY(cudaStreamWaitEvent(hp.out, hp.computed[c], 0));
+    LAMP_TRY(cudaMemcpyAsync((char*)out_host + h0 * L.oh, ws + L.o + h0 * L.oh, nh * L.oh, cudaMemcpyDeviceToHost, hp.out));
+    if (lse_host)
+      LAMP_TRY(cudaMemcpyAsync((char*)lse_host + h0 * L.lh, ws + L.lse + h0 * L.lh, nh * L.lh, cudaMemcpyDeviceToHost, hp.out));
+    if (flag_mask_host)
+      LAMP_TRY(cudaMemcpyAsync((char*)flag_mask_host + h0 * L.fh, ws + L.fm + h0 * L.fh, nh * L.fh, cudaMemcpyDeviceToHost, hp.out));
+  }
+  // the caller's stream ends the call: whatever follows on it sees the results in host memory
+  LAMP_TRY(cudaEventRecord(hp.done, hp.out));
+  LAMP_TRY(cudaStreamWaitEvent(stream, hp.done, 0));
+#undef LAMP_TRY
   return LAMP_OK;
 }
 

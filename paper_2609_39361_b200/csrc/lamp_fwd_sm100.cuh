@@ -952,8 +952,13 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
   constexpr int bq = (VAR == 4) ? 16 : kBQ;    // 32, or 16: then rows 16..31 of every group of lanes do not exist
   const int cta_rows = 4 * bq;                 // query rows of one CTA
   const int ntq = (P.seqlen + cta_rows - 1) / cta_rows;
-  const int qt = ntq - 1 - (int)blockIdx.x;   // long (late) query tiles first
-  const int h = blockIdx.y, b = blockIdx.z;
+  // blocks are handed out in index order: the query tile is the slowest index, late (long) tiles first, so the
+  // longest blocks of ALL heads start first and the launch ends on short ones; consecutive blocks are the
+  // heads of one tile, which share K and V within a group of query heads
+  const int nbh = P.heads_q * P.batch;
+  const int qt = ntq - 1 - (int)(blockIdx.x / (unsigned)nbh);
+  const int bh = (int)(blockIdx.x % (unsigned)nbh);
+  const int h = bh % P.heads_q, b = bh / P.heads_q;
   const int hk = h / (P.heads_q / P.heads_kv);
   const int m0 = qt * cta_rows;
 

@@ -313,3 +313,40 @@ def test_bad_arguments_are_rejected():
     q64 = torch.zeros(1, 2, 128, 64, device=dev, dtype=torch.bfloat16)
     with pytest.raises(lamp.LampAttnError):
         lamp.forward(q64, q64, q64)
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,N,D,flags,gr", [(2, 6, 3, 300, 128, 0, 0), (3, 8, 2, 520, 128, 0, 0), (1, 2, 1, 256, 256, 0, 0),
+                                                   (5, 4, 4, 200, 128, 8, 64), (2, 4, 2, 128, 128, 1, 16)])
+def test_host_memory_entry_point_matches_the_device_one(B, Hq, Hkv, N, D, flags, gr):
+    """Same bytes and same counters whether the tensors are given on the device or in host memory (the latter is
+    cut into ranges of (batch, kv head) pairs whose copies overlap the kernels)."""
+    import paper_2609_39361_b200 as lamp
+    dev = torch.device("cuda:0")
+    cfg = li.CONFIGS[1] if D == 128 else li.CONFIGS[3]
+    q, k, v = li.make_qkv(cfg, B=B, Hq=Hq, Hkv=Hkv, N=N, seed=41)
+    sc = li.softmax_scale(D)
+    ref = lamp.forward(q.to(dev), k.to(dev), v.to(dev), scale=sc, flags=flags, group_rows=gr, out_fp32=bool(flags & 8))
+    ref_stats = lamp.lamp_attn_get_stats()
+    p = lamp.lamp_attn_default_params()
+    p.batch, p.heads_q, p.heads_kv, p.seqlen, p.head_dim = B, Hq, Hkv, N, D
+    p.scale, p.flags, p.group_rows = sc, flags, gr
+    ws = torch.empty(lamp.lamp_attn_host_workspace_bytes(p), device=dev, dtype=torch.uint8)
+    hq, hk, hv = q.pin_memory(), k.pin_memory(), v.pin_memory()
+    for with_aux in (True, False):
+        ho = torch.zeros_like(ref["out"], device="cpu").pin_memory()
+        hl = torch.zeros_like(ref["lse"], device="cpu").pin_memory() if with_aux else None
+        hf = torch.zeros_like(ref["flags"], device="cpu").pin_memory() if with_aux else None
+        for _ in range(2):          # twice: the second call reuses the workspace, streams and events
+            lamp.lamp_attn_fwd_host(hq, hk, hv, ho, hl, hf, p, ws)
+        torch.cuda.synchronize()
+        assert torch.equal(ho, ref["out"].cpu())
+        if with_aux:
+            assert torch.equal(hl, ref["lse"].cpu()) and torch.equal(hf, ref["flags"].cpu())
+        assert lamp.lamp_attn_get_stats() == ref_stats
+    # pageable host memory gives the same result
+    ho2 = torch.zeros_like(ref["out"], device="cpu")
+    lamp.lamp_attn_fwd_host(q.contiguous(), k.contiguous(), v.contiguous(), ho2, None, None, p, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(ho2, ref["out"].cpu())
+    with pytest.raises(lamp.LampAttnError):
+        lamp.lamp_attn_fwd_host(hq, hk, hv, ho, None, None, p, ws[: ws.numel() - 256])
