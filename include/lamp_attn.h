@@ -166,11 +166,11 @@ int lamp_attn_fwd(const void* q, const void* k, const void* v, void* out, float*
  *   out_host                 host, bf16 (fp32 with LAMP_OUT_FP32), contiguous; written
  *   lse_host, flag_mask_host host, contiguous, layouts as for lamp_attn_fwd; written; may be NULL
  *   p          host; sizes, thresholds, flags and group_rows as for lamp_attn_fwd; the stride fields are not
- *              read (host tensors are contiguous); LAMP_SR_E4M3 and the dbg_* outputs are not available here
+ *              read (host tensors are contiguous); the dbg_* outputs are not available here
  *   workspace  device, 256-byte aligned, at least lamp_attn_host_workspace_bytes(p) bytes (the size of all six
  *              tensors): the library allocates no device memory here either
  * The (batch, kv head) pairs are independent problems (Sec. 3.3: the heads do not interact), so the call cuts them
- * into up to 8 ranges and overlaps the host-to-device copy of one range and the device-to-host copy of another
+ * into up to 8 ranges (fewer for small problems: every launch keeps at least three blocks per SM) and overlaps the host-to-device copy of one range and the device-to-host copy of another
  * with the kernel of a third, on two streams of its own that are ordered with cuda_stream by events: the call
  * is asynchronous, work queued on cuda_stream before it has finished before the workspace is touched, and work
  * queued on cuda_stream after it (or a synchronisation of that stream) sees the complete results in host

@@ -57,6 +57,7 @@ static int cuda_fail(cudaError_t e) {
 
 struct DeviceInit {
   bool ready[64] = {};
+  int sms[64] = {};
 };
 static DeviceInit g_init;
 
@@ -114,7 +115,7 @@ static int ensure_device(int* dev_out) {
     e = cudaFuncSetAttribute(kernels[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLaunch);
     if (e != cudaSuccess) return cuda_fail(e);
   }
-  if (dev < 64) g_init.ready[dev] = true;
+  if (dev < 64) { g_init.sms[dev] = prop.multiProcessorCount; g_init.ready[dev] = true; }
   return LAMP_OK;
 }
 
@@ -203,9 +204,11 @@ static bool empty_problem(const lamp_attn_params* p) {
 }
 
 // Checks, the memsets of the outputs that need one, and the launch.  clear_stats: start the device counters
-// from zero (a call that is split into several launches clears them once).
+// from zero (a call that is split into several launches clears them once).  head0: where this launch's heads
+// start in the numbering of the whole call (the stochastic-rounding bits are a function of that number).
 static int fwd_enqueue(const void* q, const void* k, const void* v, void* out, float* lse,
-                       uint8_t* flag_mask, const lamp_attn_params* p, cudaStream_t stream, bool clear_stats) {
+                       uint8_t* flag_mask, const lamp_attn_params* p, cudaStream_t stream, bool clear_stats,
+                       int head0 = 0) {
   int rc = check_params(q, k, v, out, p);
   if (rc) return rc;
   int dev;
@@ -223,6 +226,7 @@ static int fwd_enqueue(const void* q, const void* k, const void* v, void* out, f
   P.causal = p->causal ? 1 : 0; P.window = p->window;
   P.scale = p->scale; P.tau = p->threshold; P.delta = p->delta; P.flags = p->flags; P.sr_seed = p->sr_seed;
   P.group_rows = p->group_rows ? p->group_rows : kBQ;
+  P.sr_head0 = head0;
   P.dbg_batch = p->dbg_batch; P.dbg_head = p->dbg_head;
   P.dbg_y8 = p->dbg_y8; P.dbg_e8 = p->dbg_e8;
   P.dbg_checksums = (unsigned long long*)p->dbg_checksums;
@@ -382,8 +386,8 @@ int lamp_attn_fwd_digest(const void* q, const void* k, const void* v, void* out,
 }
 
 // ---- host-memory entry point: staged through a caller-provided device workspace, copies overlapped ----
-// The (batch, kv head) pairs are independent problems, so the call is cut into up to kHostChunks ranges of
-// them: range i is copied in on one internal stream, computed on the caller's stream and copied out on a second
+// The (batch, kv head) pairs are independent problems, so a large enough call is cut into up to kHostChunks ranges
+// of them: range i is copied in on one internal stream, computed on the caller's stream and copied out on a second
 // internal stream, ordered by events only; while range i computes, range i+1 arrives and range i-1 leaves.
 struct HostPipe {
   cudaStream_t in = nullptr, out = nullptr;
@@ -427,13 +431,11 @@ int lamp_attn_fwd_host(const void* q_host, const void* k_host, const void* v_hos
                                      ? LAMP_ERR_UNSUPPORTED_SHAPE : LAMP_ERR_INVALID_ARG;
   if (empty_problem(p)) return LAMP_OK;
   if (!q_host || !k_host || !v_host || !out_host) return LAMP_ERR_INVALID_ARG;
-  if (p->dbg_y8 || p->dbg_e8 || p->dbg_checksums || (p->flags & LAMP_SR_E4M3)) return LAMP_ERR_INVALID_ARG;
+  if (p->dbg_y8 || p->dbg_e8 || p->dbg_checksums) return LAMP_ERR_INVALID_ARG;
   const HostLayout L = host_layout(p);
   if (!workspace || workspace_bytes < L.total || ((uintptr_t)workspace & 255)) return LAMP_ERR_INVALID_ARG;
   const int rep = p->heads_q / p->heads_kv;
   const long long U = (long long)p->batch * p->heads_kv;          // independent (batch, kv head) problems
-  const int chunks = (int)(U < kHostChunks ? U : kHostChunks);
-  if ((U + chunks - 1) / chunks * rep > 65535) return LAMP_ERR_UNSUPPORTED_SHAPE;
 
   // each range runs as one batch entry with (range length) kv heads over contiguous tensors
   lamp_attn_params pp = *p;
@@ -451,6 +453,14 @@ int lamp_attn_fwd_host(const void* q_host, const void* k_host, const void* v_hos
   int rc = ensure_device(&dev);
   if (rc) return rc;
   if (dev < 0 || dev >= 64) return LAMP_ERR_UNSUPPORTED_DEVICE;
+  // as many ranges as keep every launch at three or more blocks per SM (a launch is as long as its longest block
+  // at least, so small launches would cost more than the overlap gains), at most kHostChunks
+  const long long blocks = (long long)((p->seqlen + 127) / 128) * p->heads_q * p->batch;
+  long long want = blocks / (3LL * (g_init.sms[dev] > 0 ? g_init.sms[dev] : 148));
+  if (want > kHostChunks) want = kHostChunks;
+  if (want > U) want = U;
+  const int chunks = want < 1 ? 1 : (int)want;
+  if ((U + chunks - 1) / chunks * rep > 65535) return LAMP_ERR_UNSUPPORTED_SHAPE;
   std::lock_guard<std::mutex> lock(g_pipe_mutex);
   HostPipe& hp = g_pipe[dev];
   cudaError_t e;
@@ -486,7 +496,7 @@ int lamp_attn_fwd_host(const void* q_host, const void* k_host, const void* v_hos
     lamp_attn_contiguous_strides(&pp);
     rc = fwd_enqueue(ws + L.q + h0 * L.qh, ws + L.k + u0 * L.kh, ws + L.v + u0 * L.kh, ws + L.o + h0 * L.oh,
                      lse_host ? (float*)(ws + L.lse + h0 * L.lh) : nullptr,
-                     flag_mask_host ? (uint8_t*)(ws + L.fm + h0 * L.fh) : nullptr, &pp, stream, false);
+                     flag_mask_host ? (uint8_t*)(ws + L.fm + h0 * L.fh) : nullptr, &pp, stream, false, (int)h0);
     if (rc) return rc;
     LAMP_TRY(cudaEventRecord(hp.computed[c], stream));
     LAMP_TRY(cudaStreamWaitEvent(hp.out, hp.computed[c], 0));

@@ -171,6 +171,7 @@ struct KernelParams {
   uint8_t* dbg_y8;
   uint8_t* dbg_e8;
   unsigned long long* dbg_checksums;
+  int sr_head0;   // stochastic rounding: index of this launch's first (batch, head) in the whole call's numbering
 };
 
 // Counters of the last forward call (one set per device).

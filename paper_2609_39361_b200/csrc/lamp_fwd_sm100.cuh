@@ -1167,7 +1167,7 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
             uint32_t row_key[4];
 #pragma unroll
             for (int a = 0; a < 4; ++a)
-              row_key[a] = P.sr_seed ^ ((uint32_t)(b * P.heads_q + h) * kSrMulBh) ^ ((uint32_t)(j0 + 4 * qa + a) * kSrMulRow);
+              row_key[a] = P.sr_seed ^ ((uint32_t)(P.sr_head0 + b * P.heads_q + h) * kSrMulBh) ^ ((uint32_t)(j0 + 4 * qa + a) * kSrMulRow);
             const uint32_t key0 = (uint32_t)(i0 + 16 * (lane & 3)) * kSrMulKey;
             if (hh == 0) chain8_sr<QF32, true>(qh, kf, P.scale, acc, row_key, key0, hh * kHalf);
             else chain8_sr<QF32, false>(qh, kf, P.scale, acc, row_key, key0, hh * kHalf);

@@ -316,7 +316,9 @@ def test_bad_arguments_are_rejected():
 
 
 @pytest.mark.parametrize("B,Hq,Hkv,N,D,flags,gr", [(2, 6, 3, 300, 128, 0, 0), (3, 8, 2, 520, 128, 0, 0), (1, 2, 1, 256, 256, 0, 0),
-                                                   (5, 4, 4, 200, 128, 8, 64), (2, 4, 2, 128, 128, 1, 16)])
+                                                   (5, 4, 4, 200, 128, 8, 64), (2, 4, 2, 128, 128, 1, 16), (3, 4, 2, 192, 128, 64, 0),
+                                                   # enough blocks for two and for five ranges of heads (uneven ones)
+                                                   (7, 64, 16, 256, 128, 0, 0), (9, 64, 32, 512, 128, 64, 0)])
 def test_host_memory_entry_point_matches_the_device_one(B, Hq, Hkv, N, D, flags, gr):
     """Same bytes and same counters whether the tensors are given on the device or in host memory (the latter is
     cut into ranges of (batch, kv head) pairs whose copies overlap the kernels)."""
@@ -325,11 +327,11 @@ def test_host_memory_entry_point_matches_the_device_one(B, Hq, Hkv, N, D, flags,
     cfg = li.CONFIGS[1] if D == 128 else li.CONFIGS[3]
     q, k, v = li.make_qkv(cfg, B=B, Hq=Hq, Hkv=Hkv, N=N, seed=41)
     sc = li.softmax_scale(D)
-    ref = lamp.forward(q.to(dev), k.to(dev), v.to(dev), scale=sc, flags=flags, group_rows=gr, out_fp32=bool(flags & 8))
+    ref = lamp.forward(q.to(dev), k.to(dev), v.to(dev), scale=sc, flags=flags, group_rows=gr, out_fp32=bool(flags & 8), sr_seed=7)
     ref_stats = lamp.lamp_attn_get_stats()
     p = lamp.lamp_attn_default_params()
     p.batch, p.heads_q, p.heads_kv, p.seqlen, p.head_dim = B, Hq, Hkv, N, D
-    p.scale, p.flags, p.group_rows = sc, flags, gr
+    p.scale, p.flags, p.group_rows, p.sr_seed = sc, flags, gr, 7
     ws = torch.empty(lamp.lamp_attn_host_workspace_bytes(p), device=dev, dtype=torch.uint8)
     hq, hk, hv = q.pin_memory(), k.pin_memory(), v.pin_memory()
     for with_aux in (True, False):
