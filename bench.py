@@ -328,10 +328,11 @@ def main():
     achieved = fl / (kern_ms * 1e-3) / 1e12
     peak = 4.0 / MIN_SLOTS_PER_STEP * SM_COUNT * LANES_PER_SM * SM_MAX_MHZ * 1e6 / 1e12
     # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu capture summarised in
-    # profiles/lamp_fwd_sm100_config2_ncu_full.txt (algorithmic bytes: 680 MB)
+    # profiles/lamp_fwd_sm100_config2_ncu_full.txt (algorithmic bytes: 680 MB; K and V are re-read once per band of
+    # query tiles by the block order that shortens the launch's tail, at 0.2 % of the DRAM bandwidth)
     headline = (args.mode == "lamp" and not args.no_stage1 and not args.compact and not args.h16_seq and not args.sr and args.group_rows == 32 and args.tau == 0.5 and args.delta == 2.0 ** -8
                 and args.scale_mult == 1.0 and args.window == 0)
-    traffic = {2: 657.16e6}.get(cfg.index) if headline else None
+    traffic = {2: 1114.40e6}.get(cfg.index) if headline else None
     roofline = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                 "frac": achieved / peak, "traffic": traffic,
                 "note": "peak = issue-slot bound of the emulated e4m3 accumulation at 2 slots/step, "

@@ -34,6 +34,7 @@ constexpr int kConvWarp0 = 12, kConvWarps = 2, kKWarp = 14, kCtrlWarp = 15;
 constexpr int kSlots = 4;          // ring of finished chain tiles per group
 constexpr int kTimeoutCode = -4;   // LAMP_ERR_DEVICE_TIMEOUT
 constexpr int kHalf = 128;         // channels per K / V half-tile
+constexpr int kBand = 8;           // query tiles per band of the block order
 
 struct SmemLayout {
   static constexpr int kQs = 0;                                   // head_dim 128: [128][128] fp32 q*scale
@@ -952,14 +953,19 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
   constexpr int bq = (VAR == 4) ? 16 : kBQ;    // 32, or 16: then rows 16..31 of every group of lanes do not exist
   const int cta_rows = 4 * bq;                 // query rows of one CTA
   const int ntq = (P.seqlen + cta_rows - 1) / cta_rows;
-  // blocks are handed out in index order: the query tile is the slowest index, late (long) tiles first, so the
-  // longest blocks of ALL heads start first and the launch ends on short ones; consecutive blocks are the
-  // heads of one tile, which share K and V within a group of query heads
-  const int nbh = P.heads_q * P.batch;
-  const int qt = ntq - 1 - (int)(blockIdx.x / (unsigned)nbh);
-  const int bh = (int)(blockIdx.x % (unsigned)nbh);
+  // Blocks are handed out in index order.  The slowest index is a band of kBand query tiles, late (long) tiles
+  // first, so the long blocks of ALL heads start first and the launch ends on short ones (no SM idles while the
+  // last long block finishes); within a band the order is kv head, tile, query head of the group, so the blocks
+  // that run at the same time share K and V of a few kv heads, which stay in L2.
+  const int nbh = P.heads_q * P.batch, rep = P.heads_q / P.heads_kv;
+  const int band = (int)(blockIdx.x / (unsigned)(kBand * nbh));
+  const int nb = min(kBand, ntq - band * kBand);                 // tiles of this band (the last may be short)
+  const int r = (int)(blockIdx.x - (unsigned)band * (unsigned)(kBand * nbh));
+  const int kvh = r / (nb * rep), r2 = r - kvh * (nb * rep);     // kvh: (batch, kv head) flattened
+  const int qt = ntq - 1 - (band * kBand + r2 / rep);
+  const int bh = kvh * rep + r2 % rep;                           // (batch, query head) flattened
   const int h = bh % P.heads_q, b = bh / P.heads_q;
-  const int hk = h / (P.heads_q / P.heads_kv);
+  const int hk = h / rep;
   const int m0 = qt * cta_rows;
 
   int t_begin = 0, t_end = (P.seqlen + kTK - 1) / kTK;
