@@ -49,17 +49,10 @@ typedef enum lamp_attn_error {
                                       key tile), the sub-blocks still held in 8 bits are recomputed too, under
                                       the rule of stage-2 recomputations (running maxima unchanged); they are
                                       reported in bits 4-7 of the flag byte and counted in stage2_flagged   */
-
-/* Problem statement of Algorithm 1: Q, K, V per head in HBM, safety margin
- * delta of eq. (7), threshold tau of eq. (8).  Layout: element strides for
- * (batch, head, token); the head_dim stride is 1.  Every row start must be
- * 16-byte aligned (strides multiples of 8 elements, base pointers 16-byte
- * aligned). */
 #define LAMP_H16_SEQ         0x20u /* 16-bit logits by the recursion of Sec. 4.1, c <- round_e4m11(c + k q) on
                                       the pre-scaled query, every partial sum rounded, instead of the exact dot
                                       product rounded once (the library's default reading of the 16-bit
                                       accumulation); much slower on this GPU, for comparison only          */
-
 #define LAMP_SR_E4M3         0x40u /* stochastic instead of nearest-even rounding in the 8-bit accumulation, which
                                       Sec. 3.3 proposes against swamping.  Rule (integer arithmetic, so that two
                                       implementations agree bit for bit): the fp32 bit pattern of the magnitude plus
@@ -69,6 +62,11 @@ typedef enum lamp_attn_error {
                                       (sr_seed, batch * heads_q + head, query row, key, channel).  About seven
                                       times the work per step; not combinable with LAMP_H16_SEQ               */
 
+/* Problem statement of Algorithm 1: Q, K, V per head in HBM, safety margin
+ * delta of eq. (7), threshold tau of eq. (8).  Layout: element strides for
+ * (batch, head, token); the head_dim stride is 1.  Every row start must be
+ * 16-byte aligned (strides multiples of 8 elements, base pointers 16-byte
+ * aligned). */
 typedef struct lamp_attn_params {
   int32_t batch, heads_q, heads_kv; /* heads_q % heads_kv == 0 (grouped-query attention)      */
   int32_t seqlen;                   /* any length >= 1; rows and keys past it do not exist.  In the
