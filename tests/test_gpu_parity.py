@@ -352,3 +352,40 @@ def test_host_memory_entry_point_matches_the_device_one(B, Hq, Hkv, N, D, flags,
     assert torch.equal(ho2, ref["out"].cpu())
     with pytest.raises(lamp.LampAttnError):
         lamp.lamp_attn_fwd_host(hq, hk, hv, ho, None, None, p, ws[: ws.numel() - 256])
+
+
+def _random_case(rng, nmax):
+    """One valid combination of shape, mask, thresholds and mode bits."""
+    D = int(rng.choice([128, 128, 128, 256]))
+    Hkv = int(rng.choice([1, 2]))
+    rep = int(rng.choice([1, 2, 4]))
+    bq = int(rng.choice([32, 32, 16, 64]))
+    base = [0, 0, oracle.FORCE_8BIT, oracle.FORCE_16BIT, oracle.NO_STAGE1, oracle.COMPACT_BRANCH,
+            oracle.COMPACT_BRANCH | oracle.NO_STAGE1]
+    if bq == 32:
+        base += [oracle.H16_SEQ, oracle.SR_E4M3, oracle.SR_E4M3 | oracle.COMPACT_BRANCH, oracle.H16_SEQ | oracle.NO_STAGE1]
+    flags = int(rng.choice(base))
+    causal = bool(rng.random() < 0.75)
+    window = int(rng.choice([0, 0, 40, 130])) if causal else 0
+    return dict(B=int(rng.choice([1, 2])), Hq=Hkv * rep, Hkv=Hkv, N=int(rng.integers(1, nmax)), D=D, bq=bq, flags=flags,
+                causal=causal, window=window, tau=float(rng.choice([1.0, 0.5, 0.25, 0.0625])),
+                delta=float(rng.choice([2.0 ** -8, 2.0 ** -4, 0.0])), mult=float(rng.choice([0.5, 1.0, 1.0, 3.0])),
+                sr_seed=int(rng.integers(0, 2 ** 32)))
+
+
+@pytest.mark.parametrize("case", range(48))
+def test_random_combinations(case):
+    """Seeded random draws over shapes, masks, thresholds, margins, scales, group sizes and mode bits: the
+    interactions the hand-picked cases may have missed.  Everything is compared (flags, checksums of every logit
+    and exponential byte, the dense bytes of one head, O, lse, counters)."""
+    rng = np.random.default_rng(7000 + case)
+    c = _random_case(rng, 420 if case < 24 else 900)     # the longer ones span several 128-row blocks
+    cfg = li.CONFIGS[1 if c["D"] == 128 else 3]
+    q, k, v = li.make_qkv(cfg, B=c["B"], Hq=c["Hq"], Hkv=c["Hkv"], N=c["N"], seed=7000 + case)
+    sc = li.softmax_scale(cfg.D, c["mult"])
+    kw = dict(scale=sc, causal=c["causal"], window=c["window"], flags=c["flags"], delta=c["delta"], sr_seed=c["sr_seed"])
+    ref = oracle.run_all(q, k, v, tau=c["tau"], group_rows=c["bq"], dumps=True, **kw)
+    db, dh = c["B"] - 1, c["Hq"] - 1
+    gpu = run_gpu(q, k, v, threshold=c["tau"], group_rows=c["bq"], dump=(db, dh), **kw)
+    compare_units(gpu, ref, check_stats=True, label=str(c), bq=c["bq"], allow_degenerate=bool(c["flags"] & oracle.NO_STAGE1))
+    compare_dense_bytes(gpu, ref, db, dh, bq=c["bq"])
