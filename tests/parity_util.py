@@ -9,6 +9,15 @@ REL_FRO = 1e-4      # relative Frobenius error of O and of LSE (fp32 before the 
 MAX_ABS = 1e-3      # maximum absolute error of O and of LSE
 
 
+def _e4m3_values():
+    """Value of every e4m3 byte as the oracle decodes it (0x7F, the marker of an invisible pair: -inf)."""
+    dec = oracle.lib().lamp_oracle_dec_e4m3
+    return np.array([-np.inf if b == 0x7F else dec(b) for b in range(256)])
+
+
+_E4M3_VALUE = _e4m3_values()
+
+
 def run_gpu(q, k, v, *, dump=None, checksums=True, **kw):
     dev = torch.device("cuda:0")
     res = lamp.forward(q.to(dev), k.to(dev), v.to(dev), out_fp32=True, dump=dump,
@@ -42,6 +51,14 @@ def compare_units(gpu, ref, *, check_stats=False, label="", bq=32, allow_degener
         deg = np.isneginf(rl)
         assert allow_degenerate or not deg.any(), f"{label} zero normaliser with stage 1 on at unit {(b, h, g)}"
         assert np.array_equal(np.isneginf(gl), deg), f"{label} rows with a zero normaliser differ at unit {(b, h, g)}"
+        if allow_degenerate and ref.y8 is not None:
+            # the same mechanism can leave the normaliser in the fp32 subnormal range (lse - running maximum below
+            # ln 2^-126; without stage 1 the running maximum is the largest 8-bit logit): lse is still compared,
+            # the output row holds only the few bits of a subnormal and is not
+            mu8 = _E4M3_VALUE[ref.y8[n][:nr]].max(axis=1)
+            sub = ~deg & (rl - mu8 < -126.0 * np.log(2.0))
+            assert np.array_equal(gl[sub], rl[sub]), f"{label} lse of rows with a subnormal normaliser at unit {(b, h, g)}"
+            deg = deg | sub
         go, ro, gl, rl = go[~deg], ro[~deg], gl[~deg], rl[~deg]
         worst["degenerate_rows"] = worst.get("degenerate_rows", 0) + int(deg.sum())
         if go.size == 0:
