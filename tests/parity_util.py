@@ -48,9 +48,12 @@ def compare_units(gpu, ref, *, check_stats=False, label="", bq=32, allow_degener
         # Degenerate rows: with stage 1 switched off, a stage-2 recomputation can replace the exponential of the
         # row's 8-bit maximum (1.0) by a 16-bit one that underflows, and the normaliser becomes 0: lse = -inf and
         # the output row is 0/0.  Both sides must hit the same rows; their outputs are not compared.
-        deg = np.isneginf(rl)
-        assert allow_degenerate or not deg.any(), f"{label} zero normaliser with stage 1 on at unit {(b, h, g)}"
-        assert np.array_equal(np.isneginf(gl), deg), f"{label} rows with a zero normaliser differ at unit {(b, h, g)}"
+        # (Or the opposite: a recomputed logit so far above the stale 8-bit maximum that its exponential, which has
+        # no upper clamp, overflows fp32: lse = +inf.)
+        deg = np.isinf(rl)
+        assert allow_degenerate or not deg.any(), f"{label} zero or infinite normaliser with stage 1 on at unit {(b, h, g)}"
+        assert np.array_equal(np.isinf(gl), deg) and np.array_equal(gl[deg], rl[deg]), \
+            f"{label} rows with a zero or infinite normaliser differ at unit {(b, h, g)}"
         if allow_degenerate and ref.y8 is not None:
             # the same mechanism can leave the normaliser in the fp32 subnormal range (lse - running maximum below
             # ln 2^-126; without stage 1 the running maximum is the largest 8-bit logit): lse is still compared,
