@@ -18,10 +18,27 @@ def _e4m3_values():
 _E4M3_VALUE = _e4m3_values()
 
 
-def run_gpu(q, k, v, *, dump=None, checksums=True, **kw):
+def _relayout(q, k, v, layout):
+    """The same values behind other strides (device tensors in, views out)."""
+    if layout == "bnhd":         # [B, N, H, D] storage, the layout projection layers write
+        return tuple(x.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3) for x in (q, k, v))
+    if layout == "padded":       # rows padded by 16 elements
+        def pad(x):
+            buf = torch.zeros(*x.shape[:3], x.shape[3] + 16, device=x.device, dtype=x.dtype)
+            buf[..., : x.shape[3]] = x
+            return buf[..., : x.shape[3]]
+        return pad(q), pad(k), pad(v)
+    if layout == "kv_packed":    # K and V interleaved per token in one buffer
+        kvb = torch.stack((k, v), dim=3).contiguous()          # [B, Hkv, N, 2, D]
+        return q, kvb[:, :, :, 0, :], kvb[:, :, :, 1, :]
+    assert layout == "contiguous"
+    return q, k, v
+
+
+def run_gpu(q, k, v, *, dump=None, checksums=True, layout="contiguous", **kw):
     dev = torch.device("cuda:0")
-    res = lamp.forward(q.to(dev), k.to(dev), v.to(dev), out_fp32=True, dump=dump,
-                       checksums=checksums, **kw)
+    qd, kd, vd = _relayout(q.to(dev), k.to(dev), v.to(dev), layout)
+    res = lamp.forward(qd, kd, vd, out_fp32=True, dump=dump, checksums=checksums, **kw)
     stats = lamp.lamp_attn_get_stats()
     out = {k_: (v_.cpu().numpy() if isinstance(v_, torch.Tensor) else v_) for k_, v_ in res.items()}
     out["stats"] = stats

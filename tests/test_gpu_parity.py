@@ -370,12 +370,12 @@ def _random_case(rng, nmax):
     return dict(B=int(rng.choice([1, 2])), Hq=Hkv * rep, Hkv=Hkv, N=int(rng.integers(1, nmax)), D=D, bq=bq, flags=flags,
                 causal=causal, window=window, tau=float(rng.choice([1.0, 0.5, 0.25, 0.0625])),
                 delta=float(rng.choice([2.0 ** -8, 2.0 ** -4, 0.0])), mult=float(rng.choice([0.5, 1.0, 1.0, 3.0])),
-                sr_seed=int(rng.integers(0, 2 ** 32)))
+                sr_seed=int(rng.integers(0, 2 ** 32)), layout=str(rng.choice(["contiguous", "bnhd", "padded", "kv_packed"])))
 
 
 @pytest.mark.parametrize("case", range(48))
 def test_random_combinations(case):
-    """Seeded random draws over shapes, masks, thresholds, margins, scales, group sizes and mode bits: the
+    """Seeded random draws over shapes, memory layouts, masks, thresholds, margins, scales, group sizes and mode bits: the
     interactions the hand-picked cases may have missed.  Everything is compared (flags, checksums of every logit
     and exponential byte, the dense bytes of one head, O, lse, counters)."""
     rng = np.random.default_rng(7000 + case)
@@ -386,6 +386,6 @@ def test_random_combinations(case):
     kw = dict(scale=sc, causal=c["causal"], window=c["window"], flags=c["flags"], delta=c["delta"], sr_seed=c["sr_seed"])
     ref = oracle.run_all(q, k, v, tau=c["tau"], group_rows=c["bq"], dumps=True, **kw)
     db, dh = c["B"] - 1, c["Hq"] - 1
-    gpu = run_gpu(q, k, v, threshold=c["tau"], group_rows=c["bq"], dump=(db, dh), **kw)
+    gpu = run_gpu(q, k, v, threshold=c["tau"], group_rows=c["bq"], dump=(db, dh), layout=c["layout"], **kw)
     compare_units(gpu, ref, check_stats=True, label=str(c), bq=c["bq"], allow_degenerate=bool(c["flags"] & oracle.NO_STAGE1))
     compare_dense_bytes(gpu, ref, db, dh, bq=c["bq"])
