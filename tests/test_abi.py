@@ -27,6 +27,15 @@ def test_host_only_calls_work_without_a_device():
     assert list(p.q_strides) == [8 * 256 * 128, 256 * 128, 128]
     assert list(p.k_strides) == [4 * 256 * 128, 256 * 128, 128]
     assert lamp.lamp_attn_workspace_bytes(p) == 0
+    # staging space of the host-memory call: Q, K, V, O (bf16), lse (fp32), flag mask (one byte per 32 x 64 tile)
+    head = 256 * 128 * 2
+    assert lamp.lamp_attn_host_workspace_bytes(p) == 16 * head + 2 * 8 * head + 16 * head + 16 * 256 * 4 + 16 * 8 * 4
+    p.seqlen, p.flags, p.group_rows = 200, lamp.LAMP_OUT_FP32, 16         # ragged length, fp32 out, 16-row groups
+    al = lambda x: (x + 255) // 256 * 256
+    assert lamp.lamp_attn_host_workspace_bytes(p) == (al(16 * 200 * 128 * 2) + 2 * al(8 * 200 * 128 * 2) + al(16 * 200 * 128 * 4)
+                                                      + al(16 * 200 * 4) + al(16 * 13 * 4))
+    p.head_dim = 64
+    assert lamp.lamp_attn_host_workspace_bytes(p) == 0                    # not a supported problem
     assert lamp.lamp_attn_strerror(0) == "ok" and "shape" in lamp.lamp_attn_strerror(-2)
 
 
