@@ -35,6 +35,7 @@ constexpr int kSlots = 4;          // ring of finished chain tiles per group
 constexpr int kTimeoutCode = -4;   // LAMP_ERR_DEVICE_TIMEOUT
 constexpr int kHalf = 128;         // channels per K / V half-tile
 constexpr int kBand = 8;           // query tiles per band of the block order
+constexpr long long kL2Budget = 96ll << 20;   // bytes of K + V that may be live at once (the L2 holds 126 MB)
 
 struct SmemLayout {
   static constexpr int kQs = 0;                                   // head_dim 128: [128][128] fp32 q*scale
@@ -957,12 +958,14 @@ lamp_fwd_sm100(const __grid_constant__ KernelParams P, const __grid_constant__ C
   // first, so the long blocks of ALL heads start first and the launch ends on short ones (no SM idles while the
   // last long block finishes); within a band the order is kv head, tile, query head of the group, so the blocks
   // that run at the same time share K and V of a few kv heads, which stay in L2.
+  // (When all of K and V fits in L2 with room to spare there is nothing to keep together: bands of one tile.)
   const int nbh = P.heads_q * P.batch, rep = P.heads_q / P.heads_kv;
-  const int band = (int)(blockIdx.x / (unsigned)(kBand * nbh));
-  const int nb = min(kBand, ntq - band * kBand);                 // tiles of this band (the last may be short)
-  const int r = (int)(blockIdx.x - (unsigned)band * (unsigned)(kBand * nbh));
+  const int kband = (long long)P.batch * P.heads_kv * P.seqlen * (4 * D) <= kL2Budget ? 1 : kBand;
+  const int band = (int)(blockIdx.x / (unsigned)(kband * nbh));
+  const int nb = min(kband, ntq - band * kband);                 // tiles of this band (the last may be short)
+  const int r = (int)(blockIdx.x - (unsigned)band * (unsigned)(kband * nbh));
   const int kvh = r / (nb * rep), r2 = r - kvh * (nb * rep);     // kvh: (batch, kv head) flattened
-  const int qt = ntq - 1 - (band * kBand + r2 / rep);
+  const int qt = ntq - 1 - (band * kband + r2 / rep);
   const int bh = kvh * rep + r2 % rep;                           // (batch, query head) flattened
   const int h = bh % P.heads_q, b = bh / P.heads_q;
   const int hk = h / rep;
