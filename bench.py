@@ -224,6 +224,9 @@ def main():
                     help="b_q: query rows that decide together (the paper fixes only b_q N_q = 128)")
     ap.add_argument("--scale-mult", type=float, default=1.0, help="softmax scale = mult / sqrt(head_dim)")
     ap.add_argument("--window", type=int, default=0, help="sliding window (0 = global causal)")
+    ap.add_argument("--e2e-serial", action="store_true",
+                    help="end-to-end leg as copy in, one launch, copy out (for comparison with the library's "
+                         "overlapped host-memory call, which is the default)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -298,6 +301,11 @@ def main():
     ws = torch.empty(lamp.lamp_attn_host_workspace_bytes(p), device=dev, dtype=torch.uint8)
 
     def e2e_step():
+        if args.e2e_serial:
+            dq.copy_(hq, non_blocking=True); dk.copy_(hk, non_blocking=True); dv.copy_(hv, non_blocking=True)
+            step()
+            ho.copy_(out, non_blocking=True); hl.copy_(lse, non_blocking=True); hf.copy_(fm, non_blocking=True)
+            return
         # the library's host-memory call: Q, K, V from page-locked host memory, O, lse and the flag mask back to it,
         # the copies of one range of heads overlapped with the kernel of another
         lamp.lamp_attn_fwd_host(hq, hk, hv, ho, hl, hf, p, ws)
@@ -361,7 +369,8 @@ def main():
             "dtype": "e4m3-emulated/f32", "data": "synthetic", "config": workload_config(cfg, args),
             "mode": args.mode, "clocks": clk.summary(),
             "e2e": {"value": whole_job_tflops(fl, world, e2e_ms), "unit": "TFLOP/s",
-                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
+                    "path": "copy in, one launch, copy out" if args.e2e_serial else "lamp_attn_fwd_host (overlapped)"},
             "gpu_launches": args.steps,
             "roofline": roofline, "cpu_baseline": cpu,
             "recomputed_subblock_pct": 100.0 * (stats["stage1_flagged"] + stats["stage2_flagged"]) / act,
