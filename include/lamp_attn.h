@@ -151,7 +151,8 @@ size_t lamp_attn_workspace_bytes(const lamp_attn_params* p);
  * stage-2 recomputation can leave a row with normaliser 0 (Alg. 1 keeps the running maximum in stage 2), and that
  * row gets lse = -inf and non-finite, unspecified values in out (a normaliser that lands in the fp32 subnormal range
  * leaves an output row with only a few significant bits; a recomputed logit more than 88 above the stale maximum
- * overflows its exponential, which has no upper clamp: lse = +inf).  batch = 0 or seqlen = 0 is an
+ * overflows its exponential, which has no upper clamp: lse = +inf; in the later tiles of its group such a row states
+ * no constraint in eq. (8)).  batch = 0 or seqlen = 0 is an
  * empty problem: LAMP_OK, nothing is enqueued and no pointer is looked at.
  * The call enqueues a few memsets and one kernel on the stream and nothing else, so after one call on the
  * device outside any capture (the one-time set-up) it may be recorded in a CUDA graph; a replay reads and

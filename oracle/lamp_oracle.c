@@ -202,6 +202,8 @@ static uint32_t stage2_rows(const double* xi, int ld, int nrows, const float* om
       if ((r & ~free_mask) != 0 || __builtin_popcount(r) != size) continue;
       int ok = 1;
       for (int j = 0; j < nrows && ok; ++j) {
+        /* a row whose omega_hat has overflowed (or is 0 * inf) states no constraint: eq. (8) has no meaning for it */
+        if (!isfinite(omega_hat[j])) continue;
         double kept = 0.0;
         for (int th = 0; th < NK; ++th)
           if (((free_mask & ~r) >> th) & 1u) kept += xi[th * ld + j];

@@ -835,6 +835,7 @@ __device__ __forceinline__ uint32_t lamp_post(const KernelParams& P, const TileG
       for (int th = 0; th < 4; ++th) x[th] = shfl_d(xi[a], (lane & ~3) | th);
       const double oh = (double)omh[a];
       const double rhs = __dmul_rn(__dmul_rn((double)P.tau, oh), oh);
+      if (!isfinite(omh[a])) continue;   // an overflowed normaliser states no constraint (the shortcut above agrees)
 #pragma unroll 1
       for (uint32_t r = 0; r < 16; ++r) {
         const uint32_t keep = freem & ~r;

@@ -275,6 +275,21 @@ def test_stage2_hand_example_and_tie_rule():
     assert stage2(xi, np.ones(32), 0.5, 0b1101) == 0            # 0.05+0.3+0.05 <= 0.5
 
 
+def test_stage2_ignores_rows_whose_normaliser_is_not_finite():
+    """Eq. (8) says nothing for a row whose normaliser has overflowed (possible only with stage 1 off): such a row
+    states no constraint, whatever its sums are (they are inf or NaN then), and the answer is the one of the other rows."""
+    xi = np.zeros((4, 32)); xi[:, 0] = [0.05, 0.3, 0.3, 0.05]
+    om = np.ones(32, np.float32)
+    want = stage2(xi, om, 0.5, 0b1111)
+    for bad_om, bad_xi in ((np.inf, np.nan), (np.inf, np.inf), (np.nan, np.nan), (np.nan, 0.0)):
+        xi2, om2 = xi.copy(), om.copy()
+        om2[7] = bad_om; xi2[:, 7] = bad_xi
+        assert stage2(xi2, om2, 0.5, 0b1111) == want == 0b0010
+    xi2, om2 = xi.copy(), om.copy()
+    om2[:] = np.inf; xi2[:] = np.nan
+    assert stage2(xi2, om2, 0.5, 0b1111) == 0                    # no row states anything: nothing to recompute
+
+
 def test_stage2_is_optimal_by_brute_force():
     rng = np.random.default_rng(1)
     for _ in range(300):
