@@ -147,7 +147,8 @@ size_t lamp_attn_workspace_bytes(const lamp_attn_params* p);
  *            when that is 0)
  *   cuda_stream a cudaStream_t (NULL = the default stream)
  * Inputs must be finite.  Logits beyond +-448 saturate (counted, not an error).  Every row's normaliser is at
- * least 1 and out / lse are finite, except with LAMP_NO_STAGE1 at scales where first-pass logits saturate: there a
+ * least 1 and out / lse are finite, except where first-pass logits saturate far above the true ones (with
+ * LAMP_NO_STAGE1 from moderate scales on, otherwise only at scales where nearly every logit saturates): there a
  * stage-2 recomputation can leave a row with normaliser 0 (Alg. 1 keeps the running maximum in stage 2), and that
  * row gets lse = -inf and non-finite, unspecified values in out (a normaliser that lands in the fp32 subnormal range
  * leaves an output row with only a few significant bits; a recomputed logit more than 88 above the stale maximum

@@ -67,17 +67,21 @@ def compare_units(gpu, ref, *, check_stats=False, label="", bq=32, allow_degener
         # the output row is 0/0.  Both sides must hit the same rows; their outputs are not compared.
         # (Or the opposite: a recomputed logit so far above the stale 8-bit maximum that its exponential, which has
         # no upper clamp, overflows fp32: lse = +inf.)
-        deg = np.isinf(rl)
-        assert allow_degenerate or not deg.any(), f"{label} zero or infinite normaliser with stage 1 on at unit {(b, h, g)}"
-        assert np.array_equal(np.isinf(gl), deg) and np.array_equal(gl[deg], rl[deg]), \
-            f"{label} rows with a zero or infinite normaliser differ at unit {(b, h, g)}"
+        # (At still larger scales an infinite normaliser meets a rescale by zero: NaN.)
+        deg = ~np.isfinite(rl)
+        assert allow_degenerate or not deg.any(), f"{label} normaliser that is not finite and positive at unit {(b, h, g)}"
+        assert np.array_equal(~np.isfinite(gl), deg) and np.array_equal(gl[deg], rl[deg], equal_nan=True), \
+            f"{label} rows without a finite positive normaliser differ at unit {(b, h, g)}"
         if allow_degenerate and ref.y8 is not None:
             # the same mechanism can leave the normaliser in the fp32 subnormal range (lse - running maximum below
             # ln 2^-126; without stage 1 the running maximum is the largest 8-bit logit): lse is still compared,
             # the output row holds only the few bits of a subnormal and is not
             mu8 = _E4M3_VALUE[ref.y8[n][:nr]].max(axis=1)
             sub = ~deg & (rl - mu8 < -126.0 * np.log(2.0))
-            assert np.array_equal(gl[sub], rl[sub]), f"{label} lse of rows with a subnormal normaliser at unit {(b, h, g)}"
+            # ... and at the other end a normaliser within 2^8 of the fp32 maximum: the kernel accumulates P V in
+            # fp32 and overflows where the oracle's wider accumulator does not
+            sub |= ~deg & (rl - mu8 > 120.0 * np.log(2.0))
+            assert np.array_equal(gl[sub], rl[sub]), f"{label} lse of rows with a subnormal or nearly infinite normaliser at unit {(b, h, g)}"
             deg = deg | sub
         go, ro, gl, rl = go[~deg], ro[~deg], gl[~deg], rl[~deg]
         worst["degenerate_rows"] = worst.get("degenerate_rows", 0) + int(deg.sum())

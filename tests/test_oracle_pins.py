@@ -602,11 +602,13 @@ def test_mass_shift_bound_eq4_on_a_single_tile():
 
 def test_normaliser_is_at_least_one_unless_stage_one_is_off():
     """The element that attains a row's running maximum contributes exp(0) = 1, so the normaliser is >= 1 and lse
-    is finite and >= that maximum - in every mode that keeps the maxima consistent with the logits it exponentiates.
-    With stage 1 off, stage 2 may recompute the sub-block that holds the 8-bit maximum while the maximum itself
-    stays (the reading for stage-2 recomputations): at a scale where the 8-bit accumulator saturates at 448 while
-    the true logit is far below, every exponential of the row can underflow and the normaliser becomes 0
-    (lse = -inf, output 0/0).  A degenerate case of that ablation, not of the method."""
+    is finite - always in the pure 8-bit and the all-16-bit modes, where the maximum and the exponentials come from
+    the same logits.  In the mixed modes a stage-2 recomputation keeps the maximum (the reading for stage-2
+    recomputations) and can replace that 1 by a 16-bit exponential of a logit far below it: where the 8-bit
+    accumulator saturated at 448 high above the true logit, every exponential of the row can underflow and the
+    normaliser becomes 0 (lse = -inf, output 0/0).  Stage 1 makes that rare, because it recomputes the sub-blocks near
+    the maximum and moves the maximum with them: on these inputs at three times the scale no row is lost with stage 1
+    on, a handful with it off (at eight times the scale it happens with stage 1 on as well)."""
     cfg = li.CONFIGS[1]
     q, k, v = li.make_qkv(cfg, B=1, Hq=4, Hkv=2, N=810, seed=7025)
     sc = li.softmax_scale(cfg.D, 3.0)
