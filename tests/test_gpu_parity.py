@@ -389,3 +389,43 @@ def test_random_combinations(case):
     gpu = run_gpu(q, k, v, threshold=c["tau"], group_rows=c["bq"], dump=(db, dh), layout=c["layout"], **kw)
     compare_units(gpu, ref, check_stats=True, label=str(c), bq=c["bq"], allow_degenerate=bool(c["flags"] & oracle.NO_STAGE1))
     compare_dense_bytes(gpu, ref, db, dh, bq=c["bq"])
+
+
+def _random_case_wide(rng):
+    """A wider generator: thresholds from 0 to 4, margins from 0 to 2, scales from 0.1x to 8x (from nothing saturating to
+    nearly everything), windows from one token, lengths at the tile boundaries +- 1, GQA ratios 3 and 8, iid inputs."""
+    D = int(rng.choice([128, 128, 256]))
+    Hkv = int(rng.choice([1, 2, 3])); rep = int(rng.choice([1, 2, 3, 4, 8]))
+    bq = int(rng.choice([32, 32, 16, 64]))
+    base = [0, 0, 0, oracle.FORCE_8BIT, oracle.FORCE_16BIT, oracle.NO_STAGE1, oracle.COMPACT_BRANCH,
+            oracle.COMPACT_BRANCH | oracle.NO_STAGE1]
+    if bq == 32:
+        base += [oracle.H16_SEQ, oracle.SR_E4M3, oracle.SR_E4M3 | oracle.FORCE_8BIT, oracle.H16_SEQ | oracle.COMPACT_BRANCH]
+    flags = int(rng.choice(base))
+    causal = bool(rng.random() < 0.7)
+    edges = [1, 2, 15, 16, 17, 31, 32, 33, 63, 64, 65, 127, 128, 129, 191, 192, 193, 255, 256, 257, 320, 383, 384, 385]
+    N = int(rng.choice(edges)) if rng.random() < 0.5 else int(rng.integers(1, 600))
+    window = int(rng.choice([0, 0, 1, 2, 16, 17, 63, 64, 65, 100, 500])) if causal else 0
+    return dict(B=int(rng.choice([1, 2, 3])), Hq=Hkv * rep, Hkv=Hkv, N=N, D=D, bq=bq, flags=flags, causal=causal, window=window,
+                tau=float(rng.choice([0.0, 2.0 ** -10, 0.0625, 0.25, 0.5, 1.0, 4.0])),
+                delta=float(rng.choice([0.0, 2.0 ** -8, 2.0 ** -4, 0.5, 2.0])),
+                mult=float(rng.choice([0.1, 0.5, 1.0, 1.0, 2.0, 4.0, 8.0])), sr_seed=int(rng.integers(0, 2 ** 32)),
+                layout=str(rng.choice(["contiguous", "bnhd", "padded", "kv_packed"])), cfgi=int(rng.choice([0, 1, 1, 3])))
+
+
+@pytest.mark.parametrize("case", range(2500, 2564))
+def test_random_combinations_wide(case):
+    """64 draws of the wider generator, compared in everything.  At the largest scales rows without a finite positive
+    normaliser occur (see the header): both sides must produce them on the same rows with the same lse."""
+    c = _random_case_wide(np.random.default_rng(case))
+    cfg = li.CONFIGS[c["cfgi"]]
+    if cfg.D != c["D"]:
+        cfg = li.CONFIGS[1 if c["D"] == 128 else 3]
+    q, k, v = li.make_qkv(cfg, B=c["B"], Hq=c["Hq"], Hkv=c["Hkv"], N=c["N"], seed=case)
+    sc = li.softmax_scale(cfg.D, c["mult"])
+    kw = dict(scale=sc, causal=c["causal"], window=c["window"], flags=c["flags"], delta=c["delta"], sr_seed=c["sr_seed"])
+    ref = oracle.run_all(q, k, v, tau=c["tau"], group_rows=c["bq"], dumps=True, **kw)
+    db, dh = c["B"] - 1, c["Hq"] - 1
+    gpu = run_gpu(q, k, v, threshold=c["tau"], group_rows=c["bq"], dump=(db, dh), layout=c["layout"], **kw)
+    compare_units(gpu, ref, check_stats=True, label=str(c), bq=c["bq"], allow_degenerate=True)
+    compare_dense_bytes(gpu, ref, db, dh, bq=c["bq"])
